@@ -1,0 +1,158 @@
+/* qf — fake-quantization hot path for quantization-aware training on NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libqf.so. Plain C types only. Unless a parameter says otherwise, EVERY data pointer
+ * is a DEVICE pointer owned by the caller; the library never allocates or frees device memory,
+ * keeps no state between calls, and enqueues all of its work on the CUDA stream passed as
+ * `stream` (a cudaStream_t cast to void*, NULL = the legacy default stream). Calls return as soon
+ * as the work is enqueued. Scratch memory comes from the caller through `workspace` /
+ * `workspace_bytes`; qf_workspace_bytes() says how much a call needs.
+ *
+ * Error behaviour: arguments are checked on the host before anything is launched and a non-zero
+ * qf_status_t is returned with nothing enqueued. A failed launch maps to QF_ERR_CUDA. Device-side
+ * waits are bounded; one that expires records QF_ERR_TIMEOUT in the first 4 bytes of the
+ * workspace (readable with qf_read_status() after the stream has been synchronised) and the
+ * kernel returns. Inputs must be finite; NaN / Inf give unspecified, non-faulting results.
+ *
+ * Notation follows the paper (Section 3.2): a quantizer Q maps a BF16 tensor X to low-bit codes C
+ * and metadata theta (scales, offsets); Q^-1 maps (C, theta) back to a BF16 tensor X_hat whose
+ * values lie on the format's grid (Eq. quantize-dequantize). Tensors are row-major; for a linear
+ * layer X is [M,K], W is [N,K], Y is [M,N] = X_hat . W_hat^T. Quantization blocks run along the
+ * last (contiguous) dimension.
+ */
+#ifndef QF_H_
+#define QF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Quantization formats (Table "formats"): NVFP4 = E2M1 codes, blocks of 16, E4M3 block scale,
+ * FP32 tensor scale; MXFP4 = E2M1 codes, blocks of 32, E8M0 power-of-two block scale; Q4_K =
+ * unsigned 4-bit codes, 256-weight super-blocks of 8 sub-blocks, 6-bit sub-block scale and offset
+ * under FP16 super-block factors (weight-only). NONE leaves an operand unquantized. */
+typedef enum { QF_FMT_NONE = 0, QF_FMT_NVFP4 = 1, QF_FMT_MXFP4 = 2, QF_FMT_Q4_K = 3 } qf_format_t;
+
+typedef enum {
+  QF_OK = 0,
+  QF_ERR_NULL = 1,      /* a required pointer is NULL */
+  QF_ERR_SHAPE = 2,     /* negative size, or a dimension that is not a multiple of what the format / kernel needs */
+  QF_ERR_ALIGN = 3,     /* a pointer is not 16-byte aligned */
+  QF_ERR_FORMAT = 4,    /* unknown format, or a format not allowed for this operand (Q4_K activations) */
+  QF_ERR_WORKSPACE = 5, /* workspace missing or smaller than qf_workspace_bytes() */
+  QF_ERR_CUDA = 6,      /* a CUDA runtime or driver call failed */
+  QF_ERR_TIMEOUT = 7,   /* a bounded device-side wait expired (reported through the workspace status word) */
+  QF_ERR_ARCH = 8,      /* the current device is not compute capability 10.x */
+  QF_ERR_DTYPE = 9      /* unknown output dtype */
+} qf_status_t;
+
+typedef enum { QF_DT_BF16 = 0, QF_DT_F32 = 1 } qf_dtype_t;
+
+typedef enum {
+  QF_OP_QDQ = 0,
+  QF_OP_LINEAR_FWD = 1,
+  QF_OP_LINEAR_BWD = 2,
+  QF_OP_GROUPED_FWD = 3,
+  QF_OP_GROUPED_BWD = 4
+} qf_op_t;
+
+/* flags */
+#define QF_TENSOR_SCALE_GIVEN 0x1u /* qf_qdq: read *tensor_scale instead of deriving it             */
+#define QF_W_TSCALE_GIVEN 0x1u     /* linear calls: *w_tscale is an input (tied / shared scale)      */
+#define QF_A_TSCALE_GIVEN 0x2u     /* linear calls: *a_tscale is an input (running activation scale) */
+#define QF_ACCUMULATE_DW 0x4u      /* backward: dW += ... instead of dW = ... (gradient accumulation) */
+
+const char* qf_status_string(qf_status_t s);
+int qf_version(void);
+
+/* Bytes of caller-provided scratch a call needs (always a multiple of 256, never 0).
+ * op = QF_OP_QDQ: M = rows, K = cols, N ignored. Linear ops: M, N, K as in the call; for grouped ops
+ * M = rows_padded and `groups` = number of experts. */
+size_t qf_workspace_bytes(qf_op_t op, int64_t M, int64_t N, int64_t K, int groups);
+
+/* Reads the 4-byte status word at the start of a workspace (synchronises `stream` first).
+ * host_status_out is a HOST pointer. */
+qf_status_t qf_read_status(const void* workspace, void* stream, int* host_status_out);
+
+/* Quantizer interface, both halves in one pass: (C, theta) = Q(in), out = Q^-1(C, theta)
+ * (Eq. quantize-dequantize; formats Eq. nvfp4 / Eq. mxfp4 / Eq. q4k; dequantization Eq. nvfp4-dequant /
+ * Eq. mxfp4-dequant / Eq. q4k-dequant).
+ *   in           BF16 [rows, cols], cols a multiple of the block (16 / 32 / 256).
+ *   out_bf16     BF16 [rows, cols]                                   (nullable: skip the dequantized copy)
+ *   codes        rows*cols/2 bytes, two 4-bit codes per byte          (nullable)
+ *                FP4 formats: element 2j in the low nibble of byte j, element 2j+1 in the high nibble.
+ *                Q4_K: 128 bytes per super-block; in each 64-element chunk, byte l holds element l in
+ *                the low nibble and element l+32 in the high nibble.
+ *   scales       NVFP4: u8 E4M3 [rows, cols/16]; MXFP4: u8 E8M0 [rows, cols/32];
+ *                Q4_K: 16 bytes per super-block {fp16 d, fp16 dmin, 12 bytes of packed 6-bit
+ *                (scale, offset) pairs}, [rows, cols/256]              (nullable)
+ *   tensor_scale NVFP4 only, device float*: read if flags & QF_TENSOR_SCALE_GIVEN, otherwise
+ *                written with amax(in)/(6*448) (1.0 for an all-zero tensor). Required for NVFP4.
+ * At least one of out_bf16 / codes / scales must be non-NULL. rows*cols == 0 is a no-op. */
+qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, void* out_bf16,
+                   void* codes, void* scales, float* tensor_scale, uint32_t flags, void* workspace,
+                   size_t workspace_bytes, void* stream);
+
+/* Q^-1 alone (Eq. nvfp4-dequant / Eq. mxfp4-dequant / Eq. q4k-dequant): codes + scales (+ tensor scale)
+ * -> BF16 [rows, cols]. Layouts as in qf_qdq. */
+qf_status_t qf_dequant(qf_format_t fmt, const void* codes, const void* scales, const float* tensor_scale,
+                       int64_t rows, int64_t cols, void* out_bf16, void* stream);
+
+/* Tensor-wide max |x| of a BF16 tensor of n elements, written as FP32 to *amax_out (the statistic
+ * the NVFP4 tensor scale and the trainer's running activation maximum are derived from). */
+qf_status_t qf_amax(const void* in, int64_t n, float* amax_out, void* stream);
+
+/* Quantization-aware linear layer, forward (Eq. fakequant):
+ *     Y[M,N] = Q_a^-1(Q_a(X[M,K])) . Q_w^-1(Q_w(W[N,K]))^T,   BF16 operands, FP32 accumulation.
+ *   wq_fmt in {NONE, NVFP4, MXFP4, Q4_K}; aq_fmt in {NONE, NVFP4, MXFP4}.
+ *   Y is BF16 or FP32 per y_dtype. K must be a multiple of the larger block in use (and of 8);
+ *   N a multiple of 8.
+ *   w_tscale / a_tscale: NVFP4 tensor scales (device float*), given or derived per flags
+ *   (derived values are written back); ignored for other formats and may then be NULL.
+ *   a_amax_out (nullable): receives amax(X), for the trainer's running activation maximum. */
+qf_status_t qf_fq_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N,
+                             int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
+                             float* a_tscale, float* a_amax_out, uint32_t flags, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* Straight-through backward (Eq. ste, Eq. activation-ste); both quantizers act as the identity:
+ *     dX[M,K] = dY[M,N] . W_hat[N,K]            (nullable: skip)
+ *     dW[N,K] = dY[M,N]^T . X_hat[M,K]          (nullable: skip)
+ * W_hat and X_hat are recomputed from W and X exactly as in the forward. dY is never quantized.
+ * M must be a multiple of 8 when dW is requested. */
+qf_status_t qf_fq_linear_bwd(const void* dY, const void* X, const void* W, void* dX, qf_dtype_t dx_dtype,
+                             void* dW, qf_dtype_t dw_dtype, int64_t M, int64_t N, int64_t K,
+                             qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale,
+                             uint32_t flags, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Per-expert variant for mixture-of-experts layers (every expert's latent weights are trained with
+ * the same quantization-aware layer). Rows of X are sorted by expert; group_offsets is a device
+ * int32[G+1] of segment starts, each a multiple of 128 (the caller pads segments with zero rows;
+ * a zero row quantizes to a zero row in every format); rows_padded = group_offsets[G].
+ * W is [G,N,K], Y is [rows_padded,N]:  Y[r,:] = X_hat[r,:] . W_hat[g(r)]^T. */
+qf_status_t qf_fq_grouped_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype,
+                                     const int32_t* group_offsets, int G, int64_t rows_padded, int64_t N,
+                                     int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
+                                     float* a_tscale, uint32_t flags, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
+/* dX[r,:] = dY[r,:] . W_hat[g(r)]  (nullable);  dW[g] = dY[seg g]^T . X_hat[seg g], dW is [G,N,K] (nullable). */
+qf_status_t qf_fq_grouped_linear_bwd(const void* dY, const void* X, const void* W, void* dX,
+                                     qf_dtype_t dx_dtype, void* dW, qf_dtype_t dw_dtype,
+                                     const int32_t* group_offsets, int G, int64_t rows_padded, int64_t N,
+                                     int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
+                                     float* a_tscale, uint32_t flags, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
+/* Self-test hook for the hardware number-format conversions the kernels rely on: for each of n FP32
+ * inputs (device), writes the E2M1 code (low nibble) into e2m1_out[i] and the E4M3 code of |x|
+ * into e4m3_out[i] (device u8 arrays, either nullable). Used by the tests to compare the
+ * conversion instructions exhaustively with the oracle's encoders. */
+qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8_t* e4m3_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QF_H_ */

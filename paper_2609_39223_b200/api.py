@@ -1,0 +1,245 @@
+"""Thin ctypes binding over ``libqf.so`` — argument marshalling only; every step of the path runs
+in the CUDA kernels behind the C ABI declared in ``include/qf.h``. Function names match the C
+entry points. Tensors are torch CUDA tensors (used purely as device-memory handles); work is
+enqueued on torch's current stream. There is no CPU fallback: if the library cannot be loaded or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+from pathlib import Path
+
+import torch
+
+FMT_NONE, FMT_NVFP4, FMT_MXFP4, FMT_Q4_K = 0, 1, 2, 3
+DT_BF16, DT_F32 = 0, 1
+OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 3, 4
+TENSOR_SCALE_GIVEN = 0x1
+W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW = 0x1, 0x2, 0x4
+BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
+FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
+
+LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
+
+EXPORTS = [
+    "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
+    "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
+]
+
+
+class QfError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (qf_status_t={code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libqf.so, building it first if the sources are newer. Raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        from . import build as _build
+        path = _build.build()
+        L = ctypes.CDLL(str(path))
+        L.qf_status_string.restype = c_char_p
+        L.qf_status_string.argtypes = [c_int]
+        L.qf_version.restype = c_int
+        L.qf_workspace_bytes.restype = c_size_t
+        L.qf_workspace_bytes.argtypes = [c_int, c_int64, c_int64, c_int64, c_int]
+        L.qf_read_status.restype = c_int
+        L.qf_read_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_int)]
+        L.qf_qdq.restype = c_int
+        L.qf_qdq.argtypes = [c_int, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_uint32,
+                             c_void_p, c_size_t, c_void_p]
+        L.qf_dequant.restype = c_int
+        L.qf_dequant.argtypes = [c_int, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
+        L.qf_amax.restype = c_int
+        L.qf_amax.argtypes = [c_void_p, c_int64, c_void_p, c_void_p]
+        L.qf_fq_linear_fwd.restype = c_int
+        L.qf_fq_linear_fwd.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
+                                       c_void_p, c_void_p, c_void_p, c_uint32, c_void_p, c_size_t, c_void_p]
+        L.qf_fq_linear_bwd.restype = c_int
+        L.qf_fq_linear_bwd.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int64, c_int64,
+                                       c_int64, c_int, c_int, c_void_p, c_void_p, c_uint32, c_void_p, c_size_t, c_void_p]
+        L.qf_fq_grouped_linear_fwd.restype = c_int
+        L.qf_fq_grouped_linear_fwd.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int64, c_int64,
+                                               c_int64, c_int, c_int, c_void_p, c_void_p, c_uint32, c_void_p, c_size_t,
+                                               c_void_p]
+        L.qf_fq_grouped_linear_bwd.restype = c_int
+        L.qf_fq_grouped_linear_bwd.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p,
+                                               c_int, c_int64, c_int64, c_int64, c_int, c_int, c_void_p, c_void_p,
+                                               c_uint32, c_void_p, c_size_t, c_void_p]
+        L.qf_selftest_cvt.restype = c_int
+        L.qf_selftest_cvt.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().qf_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise QfError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dt(dtype: torch.dtype) -> int:
+    if dtype == torch.bfloat16:
+        return DT_BF16
+    if dtype == torch.float32:
+        return DT_F32
+    raise TypeError(f"unsupported output dtype {dtype}")
+
+
+def _bf16(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA BF16 tensor")
+    return t
+
+
+def qf_workspace_bytes(op: int, M: int, N: int, K: int, groups: int = 1) -> int:
+    return int(lib().qf_workspace_bytes(op, M, N, K, groups))
+
+
+def workspace(op: int, M: int, N: int, K: int, groups: int = 1, device="cuda") -> torch.Tensor:
+    return torch.empty(qf_workspace_bytes(op, M, N, K, groups), dtype=torch.uint8, device=device)
+
+
+def qf_read_status(ws: torch.Tensor) -> int:
+    out = c_int(0)
+    _check(lib().qf_read_status(_ptr(ws), _stream(), ctypes.byref(out)), "qf_read_status")
+    return out.value
+
+
+def scales_shape(fmt: int, rows: int, cols: int):
+    return (rows, cols // 256, 16) if fmt == FMT_Q4_K else (rows, cols // BLOCK[fmt])
+
+
+def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_scales=True, tensor_scale=None,
+           ws: torch.Tensor | None = None, out=None, codes=None, scales=None):
+    """(C, theta) = Q(x), x_hat = Q^-1(C, theta). Returns dict(out, codes, scales, tensor_scale); the
+    tensor scale (NVFP4) is a 1-element float32 CUDA tensor, read if ``tensor_scale`` is given."""
+    x = _bf16(x, "x")
+    rows, cols = x.shape
+    dev = x.device
+    if want_out and out is None:
+        out = torch.empty_like(x)
+    if want_codes and codes is None:
+        codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
+    if want_scales and scales is None:
+        scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=dev)
+    flags = 0
+    ts = None
+    if fmt == FMT_NVFP4:
+        if tensor_scale is not None:
+            ts = tensor_scale if isinstance(tensor_scale, torch.Tensor) else torch.tensor([tensor_scale], dtype=torch.float32, device=dev)
+            flags |= TENSOR_SCALE_GIVEN
+        else:
+            ts = torch.empty(1, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(OP_QDQ, rows, 0, cols, device=dev)
+    _check(lib().qf_qdq(fmt, _ptr(x), rows, cols, _ptr(out), _ptr(codes), _ptr(scales), _ptr(ts), flags, _ptr(ws),
+                        ws.numel(), _stream()), "qf_qdq")
+    return {"out": out, "codes": codes, "scales": scales, "tensor_scale": ts}
+
+
+def qf_dequant(fmt: int, codes: torch.Tensor, scales: torch.Tensor, tensor_scale, rows: int, cols: int) -> torch.Tensor:
+    out = torch.empty((rows, cols), dtype=torch.bfloat16, device=codes.device)
+    _check(lib().qf_dequant(fmt, _ptr(codes), _ptr(scales), _ptr(tensor_scale), rows, cols, _ptr(out), _stream()), "qf_dequant")
+    return out
+
+
+def qf_amax(x: torch.Tensor) -> torch.Tensor:
+    x = _bf16(x, "x")
+    out = torch.empty(1, dtype=torch.float32, device=x.device)
+    _check(lib().qf_amax(_ptr(x), x.numel(), _ptr(out), _stream()), "qf_amax")
+    return out
+
+
+def qf_fq_linear_fwd(X, W, wq_fmt: int, aq_fmt: int, *, y_dtype=torch.bfloat16, w_tscale=None, a_tscale=None,
+                     a_amax_out=None, flags: int = 0, ws=None, Y=None) -> torch.Tensor:
+    """Y = QDQ_a(X) . QDQ_w(W)^T."""
+    X, W = _bf16(X, "X"), _bf16(W, "W")
+    M, K = X.shape
+    N = W.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=y_dtype, device=X.device)
+    if ws is None:
+        ws = workspace(OP_LINEAR_FWD, M, N, K, device=X.device)
+    _check(lib().qf_fq_linear_fwd(_ptr(X), _ptr(W), _ptr(Y), _dt(Y.dtype), M, N, K, wq_fmt, aq_fmt, _ptr(w_tscale),
+                                  _ptr(a_tscale), _ptr(a_amax_out), flags, _ptr(ws), ws.numel(), _stream()),
+           "qf_fq_linear_fwd")
+    return Y
+
+
+def qf_fq_linear_bwd(dY, X, W, wq_fmt: int, aq_fmt: int, *, dx_dtype=torch.bfloat16, dw_dtype=torch.float32,
+                     want_dx=True, want_dw=True, w_tscale=None, a_tscale=None, flags: int = 0, ws=None, dX=None, dW=None):
+    """(dX, dW) with dX = dY . QDQ_w(W) and dW = dY^T . QDQ_a(X) (straight-through estimator)."""
+    dY = _bf16(dY, "dY")
+    M, N = dY.shape
+    K = (W if W is not None else X).shape[1]
+    if want_dx and dX is None:
+        dX = torch.empty((M, K), dtype=dx_dtype, device=dY.device)
+    if want_dw and dW is None:
+        dW = torch.empty((N, K), dtype=dw_dtype, device=dY.device)
+    if ws is None:
+        ws = workspace(OP_LINEAR_BWD, M, N, K, device=dY.device)
+    _check(lib().qf_fq_linear_bwd(_ptr(dY), _ptr(X), _ptr(W), _ptr(dX), _dt(dX.dtype) if dX is not None else 0, _ptr(dW),
+                                  _dt(dW.dtype) if dW is not None else 0, M, N, K, wq_fmt, aq_fmt, _ptr(w_tscale),
+                                  _ptr(a_tscale), flags, _ptr(ws), ws.numel(), _stream()), "qf_fq_linear_bwd")
+    return dX, dW
+
+
+def qf_fq_grouped_linear_fwd(X, W, group_offsets, wq_fmt: int, aq_fmt: int, *, y_dtype=torch.bfloat16, w_tscale=None,
+                             a_tscale=None, flags: int = 0, ws=None, Y=None) -> torch.Tensor:
+    X, W = _bf16(X, "X"), _bf16(W, "W")
+    rows, K = X.shape
+    G, N, _ = W.shape
+    if Y is None:
+        Y = torch.empty((rows, N), dtype=y_dtype, device=X.device)
+    if ws is None:
+        ws = workspace(OP_GROUPED_FWD, rows, N, K, G, device=X.device)
+    _check(lib().qf_fq_grouped_linear_fwd(_ptr(X), _ptr(W), _ptr(Y), _dt(Y.dtype), _ptr(group_offsets), G, rows, N, K,
+                                          wq_fmt, aq_fmt, _ptr(w_tscale), _ptr(a_tscale), flags, _ptr(ws), ws.numel(),
+                                          _stream()), "qf_fq_grouped_linear_fwd")
+    return Y
+
+
+def qf_fq_grouped_linear_bwd(dY, X, W, group_offsets, wq_fmt: int, aq_fmt: int, *, dx_dtype=torch.bfloat16,
+                             dw_dtype=torch.float32, want_dx=True, want_dw=True, w_tscale=None, a_tscale=None,
+                             flags: int = 0, ws=None, dX=None, dW=None):
+    dY = _bf16(dY, "dY")
+    rows, N = dY.shape
+    G, _, K = W.shape
+    if want_dx and dX is None:
+        dX = torch.empty((rows, K), dtype=dx_dtype, device=dY.device)
+    if want_dw and dW is None:
+        dW = torch.empty((G, N, K), dtype=dw_dtype, device=dY.device)
+    if ws is None:
+        ws = workspace(OP_GROUPED_BWD, rows, N, K, G, device=dY.device)
+    _check(lib().qf_fq_grouped_linear_bwd(_ptr(dY), _ptr(X), _ptr(W), _ptr(dX), _dt(dX.dtype) if dX is not None else 0,
+                                          _ptr(dW), _dt(dW.dtype) if dW is not None else 0, _ptr(group_offsets), G, rows,
+                                          N, K, wq_fmt, aq_fmt, _ptr(w_tscale), _ptr(a_tscale), flags, _ptr(ws),
+                                          ws.numel(), _stream()), "qf_fq_grouped_linear_bwd")
+    return dX, dW
+
+
+def qf_selftest_cvt(x: torch.Tensor):
+    """E2M1 and E4M3 codes the hardware conversion instructions produce for each FP32 input."""
+    assert x.dtype == torch.float32 and x.is_cuda and x.is_contiguous()
+    e2 = torch.empty(x.numel(), dtype=torch.uint8, device=x.device)
+    e4 = torch.empty(x.numel(), dtype=torch.uint8, device=x.device)
+    _check(lib().qf_selftest_cvt(_ptr(x), x.numel(), _ptr(e2), _ptr(e4), _stream()), "qf_selftest_cvt")
+    return e2, e4

@@ -1,0 +1,358 @@
+// C ABI of libqf.so: argument validation, workspace carving, and the launch sequences of the
+// quantizer and of the quantization-aware linear layer (forward and straight-through backward).
+// Nothing here computes; every step of the path runs in the kernels of qf_qdq.cu / qf_gemm.cu.
+#include <stdio.h>
+
+#include "qf_common.cuh"
+
+namespace qf {
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round256(size_t b) { return (b + 255) & ~static_cast<size_t>(255); }
+
+inline int block_of(int fmt) {
+  switch (fmt) {
+    case QF_FMT_NVFP4: return 16;
+    case QF_FMT_MXFP4: return 32;
+    case QF_FMT_Q4_K: return 256;
+    default: return 0;
+  }
+}
+inline bool valid_fmt(int fmt, bool allow_none) { return (fmt >= (allow_none ? 0 : 1)) && fmt <= 3; }
+
+// The device must be a compute-capability 10.x part: the kernels are built for sm_100a only.
+qf_status_t check_arch() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return QF_ERR_CUDA; }
+  static int cached_major[64] = {0};
+  int major = dev < 64 ? cached_major[dev] : 0;
+  if (major == 0) {
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) { cudaGetLastError(); return QF_ERR_CUDA; }
+    if (dev < 64) cached_major[dev] = major;
+  }
+  return major == 10 ? QF_OK : QF_ERR_ARCH;
+}
+
+inline qf_status_t cu(cudaError_t e) {
+  if (e == cudaSuccess) return QF_OK;
+  cudaGetLastError();
+  return QF_ERR_CUDA;
+}
+
+struct Workspace {
+  uint32_t* header;     // 64 words
+  uint8_t* w_hat;       // fake-quantized weights
+  uint8_t* x_hat;       // fake-quantized activations
+};
+
+size_t linear_ws_bytes(int64_t M, int64_t N, int64_t K, int64_t groups) {
+  return kWsHeader + round256(static_cast<size_t>(groups) * N * K * 2) + round256(static_cast<size_t>(M) * K * 2);
+}
+
+Workspace carve(void* ws, int64_t N, int64_t K, int64_t groups) {
+  Workspace w;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  w.header = reinterpret_cast<uint32_t*>(base);
+  w.w_hat = base + kWsHeader;
+  w.x_hat = w.w_hat + round256(static_cast<size_t>(groups) * N * K * 2);
+  return w;
+}
+
+// Fake-quantize one operand into `dst` (BF16, same shape). NVFP4 derives or reads its tensor scale.
+qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t cols, void* dst, float* tscale_user,
+                             bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st) {
+  QdqArgs q{};
+  q.fmt = fmt;
+  q.in = src;
+  q.rows = rows;
+  q.cols = cols;
+  q.out = dst;
+  if (fmt == QF_FMT_NVFP4) {
+    if (tscale_given) {
+      q.tscale_in = tscale_user;
+    } else {
+      if (cudaError_t e = launch_amax(src, rows * cols, header + amax_word, st)) return cu(e);
+      q.amax_bits = header + amax_word;
+      q.tscale_out = tscale_user ? tscale_user : reinterpret_cast<float*>(header + scale_word);
+    }
+  }
+  return cu(launch_qdq(q, st));
+}
+
+qf_status_t check_linear_common(const void* W, int64_t M, int64_t N, int64_t K, int wq, int aq, const float* w_ts,
+                                const float* a_ts, uint32_t flags, void* ws, size_t ws_bytes, int64_t groups) {
+  if (!W || !ws) return !W ? QF_ERR_NULL : QF_ERR_WORKSPACE;
+  if (M < 0 || N < 0 || K < 0) return QF_ERR_SHAPE;
+  if (!valid_fmt(wq, true) || !valid_fmt(aq, true)) return QF_ERR_FORMAT;
+  if (aq == QF_FMT_Q4_K) return QF_ERR_FORMAT;                    // Q4_K is a weight-only format
+  if (K % 8 || N % 8) return QF_ERR_SHAPE;
+  if (wq != QF_FMT_NONE && K % block_of(wq)) return QF_ERR_SHAPE;
+  if (aq != QF_FMT_NONE && K % block_of(aq)) return QF_ERR_SHAPE;
+  if (wq == QF_FMT_NVFP4 && (flags & QF_W_TSCALE_GIVEN) && !w_ts) return QF_ERR_NULL;
+  if (aq == QF_FMT_NVFP4 && (flags & QF_A_TSCALE_GIVEN) && !a_ts) return QF_ERR_NULL;
+  if (!aligned16(W) || !aligned16(ws)) return QF_ERR_ALIGN;
+  if (ws_bytes < linear_ws_bytes(M, N, K, groups)) return QF_ERR_WORKSPACE;
+  return QF_OK;
+}
+
+inline bool valid_dtype(int d) { return d == QF_DT_BF16 || d == QF_DT_F32; }
+
+// Shared by the plain and the grouped calls (groups == 1 and offs == nullptr for the plain ones).
+qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, const int32_t* offs, int G, int64_t M,
+                            int64_t N, int64_t K, int wq, int aq, float* w_ts, float* a_ts, float* a_amax_out,
+                            uint32_t flags, void* ws, size_t ws_bytes, cudaStream_t st) {
+  const bool grouped = offs != nullptr;
+  const int64_t groups = grouped ? G : 1;
+  if (!X || !Y) return QF_ERR_NULL;
+  if (!valid_dtype(y_dtype)) return QF_ERR_DTYPE;
+  if (qf_status_t s = check_linear_common(W, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
+  if (!aligned16(X) || !aligned16(Y)) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  if (M == 0 || N == 0) return QF_OK;
+  Workspace w = carve(ws, N, K, groups);
+  if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
+  const void* Wh = W;
+  const void* Xh = X;
+  if (K > 0) {
+    if (wq != QF_FMT_NONE) {
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      Wh = w.w_hat;
+    }
+    if (a_amax_out) {
+      if (cudaError_t e = launch_amax(X, M * K, w.header + 6, st)) return cu(e);
+      if (cudaError_t e = launch_amax_to_float(w.header + 6, a_amax_out, st)) return cu(e);
+    }
+    if (aq != QF_FMT_NONE) {
+      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      Xh = w.x_hat;
+    }
+  }
+  GemmArgs g{};
+  g.A = Xh; g.B = Wh; g.C = Y;
+  g.Mo = M; g.No = N; g.Kc = K;
+  g.lda = K; g.ldb = K; g.ldc = N;
+  g.a_mn_major = false; g.b_mn_major = false;
+  g.c_dtype = y_dtype;
+  g.status_word = w.header + kWsStatus;
+  if (grouped) {
+    g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M;
+  }
+  return cu(launch_gemm(g, st));
+}
+
+qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* dX, int dx_dtype, void* dW, int dw_dtype,
+                            const int32_t* offs, int G, int64_t M, int64_t N, int64_t K, int wq, int aq, float* w_ts,
+                            float* a_ts, uint32_t flags, void* ws, size_t ws_bytes, cudaStream_t st) {
+  const bool grouped = offs != nullptr;
+  const int64_t groups = grouped ? G : 1;
+  if (!dY) return QF_ERR_NULL;
+  if (!dX && !dW) return QF_ERR_NULL;
+  if (dW && !X) return QF_ERR_NULL;
+  if ((dX && !valid_dtype(dx_dtype)) || (dW && !valid_dtype(dw_dtype))) return QF_ERR_DTYPE;
+  if (qf_status_t s = check_linear_common(W ? W : dY, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
+  if (dX && !W) return QF_ERR_NULL;
+  if (!aligned16(dY) || (X && !aligned16(X)) || (dX && !aligned16(dX)) || (dW && !aligned16(dW))) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  if (M == 0 || N == 0 || K == 0) {
+    // an empty contraction still defines the outputs: they are zero (unless accumulating)
+    if (dW && M == 0 && N > 0 && K > 0 && !(flags & QF_ACCUMULATE_DW))
+      if (cudaError_t e = cudaMemsetAsync(dW, 0, static_cast<size_t>(groups) * N * K * (dw_dtype == QF_DT_F32 ? 4 : 2), st)) return cu(e);
+    if (dX && N == 0 && M > 0 && K > 0)
+      if (cudaError_t e = cudaMemsetAsync(dX, 0, static_cast<size_t>(M) * K * (dx_dtype == QF_DT_F32 ? 4 : 2), st)) return cu(e);
+    return QF_OK;
+  }
+  Workspace w = carve(ws, N, K, groups);
+  if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
+  if (dX) {
+    const void* Wh = W;
+    if (wq != QF_FMT_NONE) {
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      Wh = w.w_hat;
+    }
+    // dX[M,K] = dY[M,N] . W_hat[N,K]: A = dY contraction-major, B = W_hat stored [contraction N, K]
+    GemmArgs g{};
+    g.A = dY; g.B = Wh; g.C = dX;
+    g.Mo = M; g.No = K; g.Kc = N;
+    g.lda = N; g.ldb = K; g.ldc = K;
+    g.a_mn_major = false; g.b_mn_major = true;
+    g.c_dtype = dx_dtype;
+    g.status_word = w.header + kWsStatus;
+    if (grouped) { g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M; }
+    if (cudaError_t e = launch_gemm(g, st)) return cu(e);
+  }
+  if (dW) {
+    const void* Xh = X;
+    if (aq != QF_FMT_NONE) {
+      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      Xh = w.x_hat;
+    }
+    // dW[N,K] = dY[M,N]^T . X_hat[M,K]: both operands stored [contraction M, rows]
+    GemmArgs g{};
+    g.A = dY; g.B = Xh; g.C = dW;
+    g.Mo = N; g.No = K; g.Kc = M;
+    g.lda = N; g.ldb = K; g.ldc = K;
+    g.a_mn_major = true; g.b_mn_major = true;
+    g.c_dtype = dw_dtype;
+    g.accumulate = (flags & QF_ACCUMULATE_DW) != 0;
+    g.status_word = w.header + kWsStatus;
+    if (grouped) { g.group_mode = 2; g.group_offsets = offs; g.G = G; g.rows_padded = M; g.c_group_stride = N * K; }
+    if (cudaError_t e = launch_gemm(g, st)) return cu(e);
+  }
+  return QF_OK;
+}
+
+}  // namespace
+}  // namespace qf
+
+using namespace qf;
+
+extern "C" {
+
+const char* qf_status_string(qf_status_t s) {
+  switch (s) {
+    case QF_OK: return "ok";
+    case QF_ERR_NULL: return "a required pointer is NULL";
+    case QF_ERR_SHAPE: return "bad shape (negative, or not a multiple of the block / vector width)";
+    case QF_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case QF_ERR_FORMAT: return "unknown format, or format not allowed for this operand";
+    case QF_ERR_WORKSPACE: return "workspace missing or too small";
+    case QF_ERR_CUDA: return "CUDA call failed";
+    case QF_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case QF_ERR_ARCH: return "device is not compute capability 10.x";
+    case QF_ERR_DTYPE: return "unknown output dtype";
+  }
+  return "unknown status";
+}
+
+int qf_version(void) { return 100; }
+
+size_t qf_workspace_bytes(qf_op_t op, int64_t M, int64_t N, int64_t K, int groups) {
+  if (M < 0) M = 0;
+  if (N < 0) N = 0;
+  if (K < 0) K = 0;
+  if (op == QF_OP_QDQ) return kWsHeader;
+  const int64_t g = (op == QF_OP_GROUPED_FWD || op == QF_OP_GROUPED_BWD) ? (groups > 0 ? groups : 1) : 1;
+  return linear_ws_bytes(M, N, K, g);
+}
+
+qf_status_t qf_read_status(const void* workspace, void* stream, int* host_status_out) {
+  if (!workspace || !host_status_out) return QF_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaError_t e = cudaStreamSynchronize(st)) return cu(e);
+  uint32_t v = 0;
+  if (cudaError_t e = cudaMemcpy(&v, workspace, 4, cudaMemcpyDeviceToHost)) return cu(e);
+  *host_status_out = static_cast<int>(v);
+  return QF_OK;
+}
+
+qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, void* out_bf16, void* codes,
+                   void* scales, float* tensor_scale, uint32_t flags, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+  if (!valid_fmt(fmt, false)) return QF_ERR_FORMAT;
+  if (rows < 0 || cols < 0 || cols % block_of(fmt)) return QF_ERR_SHAPE;
+  const bool empty = rows == 0 || cols == 0;            // an empty tensor has no data pointers to check
+  if (!empty && !in) return QF_ERR_NULL;
+  if (!empty && !out_bf16 && !codes && !scales) return QF_ERR_NULL;
+  if (fmt == QF_FMT_NVFP4 && !tensor_scale) return QF_ERR_NULL;
+  if (!aligned16(in) || (out_bf16 && !aligned16(out_bf16)) || (codes && !aligned16(codes)) || (scales && !aligned16(scales)))
+    return QF_ERR_ALIGN;
+  const bool need_amax = fmt == QF_FMT_NVFP4 && !(flags & QF_TENSOR_SCALE_GIVEN);
+  if (need_amax) {
+    if (!workspace || workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QF_ERR_ALIGN;
+  }
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  QdqArgs q{};
+  q.fmt = fmt;
+  q.in = in;
+  q.rows = rows;
+  q.cols = cols;
+  q.out = out_bf16;
+  q.codes = codes;
+  q.scales = scales;
+  if (fmt == QF_FMT_NVFP4) {
+    if (need_amax) {
+      uint32_t* header = static_cast<uint32_t*>(workspace);
+      if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
+      if (cudaError_t e = launch_amax(in, rows * cols, header + kWsAmaxW, st)) return cu(e);
+      q.amax_bits = header + kWsAmaxW;
+      q.tscale_out = tensor_scale;
+    } else {
+      q.tscale_in = tensor_scale;
+    }
+  }
+  return cu(launch_qdq(q, st));
+}
+
+qf_status_t qf_dequant(qf_format_t fmt, const void* codes, const void* scales, const float* tensor_scale, int64_t rows,
+                       int64_t cols, void* out_bf16, void* stream) {
+  if (!valid_fmt(fmt, false)) return QF_ERR_FORMAT;
+  if (!codes || !scales || !out_bf16) return QF_ERR_NULL;
+  if (fmt == QF_FMT_NVFP4 && !tensor_scale) return QF_ERR_NULL;
+  if (rows < 0 || cols < 0 || cols % block_of(fmt)) return QF_ERR_SHAPE;
+  if (!aligned16(codes) || !aligned16(out_bf16) || (fmt == QF_FMT_Q4_K && !aligned16(scales))) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  return cu(launch_dequant(fmt, codes, scales, tensor_scale, rows, cols, out_bf16, static_cast<cudaStream_t>(stream)));
+}
+
+qf_status_t qf_amax(const void* in, int64_t n, float* amax_out, void* stream) {
+  if (!in || !amax_out) return QF_ERR_NULL;
+  if (n < 0) return QF_ERR_SHAPE;
+  if (!aligned16(in)) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the result word doubles as the accumulator: FP32 bits of a non-negative value
+  if (cudaError_t e = cudaMemsetAsync(amax_out, 0, 4, st)) return cu(e);
+  if (n == 0) return QF_OK;
+  return cu(launch_amax(in, n, reinterpret_cast<uint32_t*>(amax_out), st));
+}
+
+qf_status_t qf_fq_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N, int64_t K,
+                             qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale, float* a_amax_out,
+                             uint32_t flags, void* workspace, size_t workspace_bytes, void* stream) {
+  return linear_fwd_impl(X, W, Y, y_dtype, nullptr, 1, M, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale, a_amax_out, flags,
+                         workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+qf_status_t qf_fq_linear_bwd(const void* dY, const void* X, const void* W, void* dX, qf_dtype_t dx_dtype, void* dW,
+                             qf_dtype_t dw_dtype, int64_t M, int64_t N, int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt,
+                             float* w_tscale, float* a_tscale, uint32_t flags, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  return linear_bwd_impl(dY, X, W, dX, dx_dtype, dW, dw_dtype, nullptr, 1, M, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale,
+                         flags, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+static qf_status_t check_groups(const int32_t* offs, int G, int64_t rows_padded) {
+  if (!offs) return QF_ERR_NULL;
+  if (G <= 0 || rows_padded < 0 || rows_padded % 128) return QF_ERR_SHAPE;
+  return QF_OK;
+}
+
+qf_status_t qf_fq_grouped_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, const int32_t* group_offsets,
+                                     int G, int64_t rows_padded, int64_t N, int64_t K, qf_format_t wq_fmt,
+                                     qf_format_t aq_fmt, float* w_tscale, float* a_tscale, uint32_t flags, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  if (qf_status_t s = check_groups(group_offsets, G, rows_padded)) return s;
+  return linear_fwd_impl(X, W, Y, y_dtype, group_offsets, G, rows_padded, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale, nullptr,
+                         flags, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+qf_status_t qf_fq_grouped_linear_bwd(const void* dY, const void* X, const void* W, void* dX, qf_dtype_t dx_dtype, void* dW,
+                                     qf_dtype_t dw_dtype, const int32_t* group_offsets, int G, int64_t rows_padded, int64_t N,
+                                     int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale,
+                                     uint32_t flags, void* workspace, size_t workspace_bytes, void* stream) {
+  if (qf_status_t s = check_groups(group_offsets, G, rows_padded)) return s;
+  return linear_bwd_impl(dY, X, W, dX, dx_dtype, dW, dw_dtype, group_offsets, G, rows_padded, N, K, wq_fmt, aq_fmt, w_tscale,
+                         a_tscale, flags, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8_t* e4m3_out, void* stream) {
+  if (!in || (!e2m1_out && !e4m3_out)) return QF_ERR_NULL;
+  if (n < 0) return QF_ERR_SHAPE;
+  if (qf_status_t s = check_arch()) return s;
+  return cu(launch_selftest_cvt(in, n, e2m1_out, e4m3_out, static_cast<cudaStream_t>(stream)));
+}
+
+}  // extern "C"

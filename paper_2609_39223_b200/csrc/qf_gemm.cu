@@ -1,0 +1,519 @@
+// BF16 x BF16 -> FP32 matmul on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory), operands staged by TMA into 128-byte-swizzled shared memory. One persistent CTA
+// per SM walks output tiles of 128 x 256; a 4-stage TMA ring feeds a single MMA-issuing thread;
+// the 512 TMEM columns hold two accumulators so the epilogue of one tile overlaps the main loop of
+// the next.
+//
+// The three products of the quantization-aware layer (Eq. fakequant, Eq. ste, Eq. activation-ste)
+// differ only in which operand dimension is contiguous in memory:
+//   forward  Y  = X_hat . W_hat^T : both operands contraction-major ("K-major")
+//   dgrad    dX = dY . W_hat      : A contraction-major, B row-major over the contraction ("MN-major")
+//   wgrad    dW = dY^T . X_hat    : both MN-major
+// so one kernel, templated on the two majors, serves all of them; the shared-memory descriptor and
+// the TMA box shape change, the pipeline does not.
+//
+// Every wait on an mbarrier is bounded. A wait that gives up raises a CTA-wide abort flag and
+// records QF_ERR_TIMEOUT in the caller's status word; all roles then fall through to the common
+// teardown (the producer first gives its outstanding copies a bounded chance to land), tensor
+// memory is released and the kernel returns.
+#include <cuda.h>
+
+#include "qf_common.cuh"
+
+namespace qf {
+namespace {
+
+constexpr int BM = 128;                 // output rows per tile   (UMMA M)
+constexpr int BN = 256;                 // output cols per tile   (UMMA N)
+constexpr int BK = 64;                  // contraction per stage  (one 128-byte swizzle row of BF16)
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;    // 16 KB
+constexpr int B_BYTES = BN * BK * 2;    // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int ACC_COLS = BN;            // FP32 accumulator columns per tile
+constexpr int TMEM_COLS = 2 * ACC_COLS; // 512: two accumulators
+constexpr int NUM_THREADS = 192;        // warp 0 TMA, warp 1 MMA + TMEM owner, warps 2-5 epilogue
+constexpr int EPI_THREADS = 128;
+constexpr long long kWaitCycles = 1ll << 31; // SM clock cycles (about a second) before a wait gives up
+
+struct alignas(8) Barriers {
+  uint64_t full[STAGES];
+  uint64_t empty[STAGES];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* Barriers */;
+
+struct KParams {
+  void* C;
+  int64_t Mo, No, Kc, ldc;
+  int c_dtype, accumulate;
+  int tiles_m, tiles_n, num_tiles;
+  int group_mode, G;
+  const int32_t* offs;
+  int64_t b_group_rows;      // mode 1: rows one group occupies in B's 2-D tensor map
+  int64_t c_group_stride;    // mode 2: elements between per-group outputs
+  uint32_t* status;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait. Returns false if the CTA is aborting (this wait or another one gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xFFu) == 0xFFu) {
+      if (*abort_flag) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitCycles) break;
+    }
+  }
+  *abort_flag = 1;
+  if (status) atomicExch(status, static_cast<uint32_t>(QF_ERR_TIMEOUT));
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the mbarrier once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- descriptors ------------------------------------------------------------------------------
+
+// Shared-memory matrix descriptor, 128-byte swizzle. Offsets are in 16-byte units.
+//   contraction-major tile: rows of 128 bytes, 8-row groups 1024 bytes apart (stride offset);
+//     the leading offset is not used by the hardware for this layout.
+//   MN-major tile: TMA boxes of 64 (MN) x 64 (contraction) elements = 8 KB each; inside a box the
+//     8-row contraction groups are 1024 bytes apart (stride offset) and successive 64-element MN
+//     groups are one box = 8192 bytes apart (leading offset).
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  const uint64_t lbo = MN_MAJOR ? (8192u >> 4) : 1u;
+  const uint64_t sbo = 1024u >> 4;
+  return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+// 16-byte units to advance the start address by for the next 16 contraction elements
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint32_t desc_k_step() { return MN_MAJOR ? (UMMA_K * 128u) >> 4 : (UMMA_K * 2u) >> 4; }
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ uint32_t instr_desc() {
+  return (1u << 4)                      // D = FP32
+         | (1u << 7) | (1u << 10)       // A, B = BF16
+         | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16)
+         | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+}
+
+// ---- tile bookkeeping ---------------------------------------------------------------------------
+
+struct Tile {
+  int m0, n0;          // output coordinates (rows of A, rows of B)
+  int k_begin, k_end;  // contraction range
+  int b_row_off;       // mode 1: row offset of this tile's group in B's tensor map
+  int64_t c_off;       // mode 2: element offset of this tile's group in C
+  int m_limit;         // rows of C that exist for this tile's matrix
+};
+
+__device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_group) {
+  Tile r;
+  r.b_row_off = 0;
+  r.c_off = 0;
+  r.k_begin = 0;
+  r.k_end = static_cast<int>(p.Kc);
+  r.m_limit = static_cast<int>(p.Mo);
+  int g = 0;
+  if (p.group_mode == 2) {
+    const int per = p.tiles_m * p.tiles_n;
+    g = t / per;
+    t -= g * per;
+  }
+  // m fastest inside bands of 8 row-tiles: concurrently running CTAs share A and B tiles in L2
+  const int band = 8 * p.tiles_n;
+  const int bidx = t / band;
+  const int first_m = bidx * 8;
+  const int rows_in_band = min(8, p.tiles_m - first_m);
+  const int within = t - bidx * band;
+  r.m0 = (first_m + within % rows_in_band) * BM;
+  r.n0 = (within / rows_in_band) * BN;
+  if (p.group_mode == 1 && need_group) {
+    // segments start on multiples of BM, so a row tile lies in exactly one group: find it
+    int lo = 0, hi = p.G;                   // invariant: offs[lo] <= m0 < offs[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(p.offs + mid) <= r.m0) lo = mid; else hi = mid;
+    }
+    r.b_row_off = lo * static_cast<int>(p.b_group_rows);
+  } else if (p.group_mode == 2) {
+    r.k_begin = __ldg(p.offs + g);
+    r.k_end = __ldg(p.offs + g + 1);
+    r.c_off = static_cast<int64_t>(g) * p.c_group_stride;
+  }
+  return r;
+}
+
+// ---- epilogue stores ------------------------------------------------------------------------------
+
+template <typename OutT>
+__device__ __forceinline__ void store_chunk32(OutT* row_ptr, int col0, int n_limit, const uint32_t (&acc)[32], bool accumulate);
+
+template <>
+__device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* row_ptr, int col0, int n_limit,
+                                                             const uint32_t (&acc)[32], bool accumulate) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const int col = col0 + 8 * g;
+    if (col + 8 <= n_limit) {
+      uint4* dst = reinterpret_cast<uint4*>(row_ptr + col);
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(acc[8 * g + j]);
+      if (accumulate) {
+        const uint4 old = *dst;
+        const uint32_t w[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] += bf16_lo(w[j]);
+          v[2 * j + 1] += bf16_hi(w[j]);
+        }
+      }
+      *dst = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+    }
+  }
+}
+
+template <>
+__device__ __forceinline__ void store_chunk32<float>(float* row_ptr, int col0, int n_limit, const uint32_t (&acc)[32],
+                                                     bool accumulate) {
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    const int col = col0 + 4 * g;
+    if (col + 4 <= n_limit) {
+      float4* dst = reinterpret_cast<float4*>(row_ptr + col);
+      float4 v = make_float4(__uint_as_float(acc[4 * g]), __uint_as_float(acc[4 * g + 1]), __uint_as_float(acc[4 * g + 2]),
+                             __uint_as_float(acc[4 * g + 3]));
+      if (accumulate) {
+        const float4 old = *dst;
+        v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+      }
+      *dst = v;
+    }
+  }
+}
+
+// ---- the kernel -----------------------------------------------------------------------------------
+
+template <bool A_MN, bool B_MN, typename OutT>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;                   // swizzled tiles need 1024-byte alignment
+  uint8_t* tiles_ptr = smem_raw + (tiles_base - raw);
+  Barriers* bars = reinterpret_cast<Barriers*>(tiles_ptr + STAGES * STAGE_BYTES);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), EPI_THREADS);
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ===== TMA producer =====
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued = 0;
+      bool alive = true;
+      for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+        const Tile tile = decode_tile(p, t, true);
+        for (int k = tile.k_begin; k < tile.k_end; k += BK) {
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status)) { alive = false; break; }
+          const uint32_t full = smem_u32(&bars->full[stage]);
+          const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          mbar_expect_tx(full, STAGE_BYTES);
+          if (A_MN) {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * 8192, &tmA, tile.m0 + 64 * i, k, full);
+          } else {
+            tma_load_2d(a_dst, &tmA, k, tile.m0, full);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmB, tile.n0 + 64 * i, tile.b_row_off + k, full);
+          } else {
+            tma_load_2d(b_dst, &tmB, k, tile.b_row_off + tile.n0, full);
+          }
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!alive) {
+        // give copies already in flight a bounded chance to land before the CTA retires
+        uint32_t s = stage, ph = phase;
+        for (uint32_t n = 0; n < min(issued, static_cast<uint32_t>(STAGES)); ++n) {
+          if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+          for (uint32_t it = 0; it < (1u << 16); ++it)
+            if (mbar_try_wait(smem_u32(&bars->full[s]), ph)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer =====
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc<A_MN, B_MN>();
+      uint32_t stage = 0, phase = 0;
+      uint32_t local = 0;
+      bool alive = true;
+      for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x, ++local) {
+        const Tile tile = decode_tile(p, t, false);
+        const uint32_t buf = local & 1u;
+        const uint32_t use = local >> 1;                      // how many times this accumulator was used before
+        if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), (use & 1u) ^ 1u, abort_flag, p.status)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
+        uint32_t accumulate = 0;
+        for (int k = tile.k_begin; k < tile.k_end; k += BK) {
+          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
+          const uint64_t a_desc = smem_desc<A_MN>(a_addr);
+          const uint64_t b_desc = smem_desc<B_MN>(a_addr + A_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            umma_bf16(d_tmem, a_desc + kk * desc_k_step<A_MN>(), b_desc + kk * desc_k_step<B_MN>(), idesc, accumulate);
+            accumulate = 1;
+          }
+          umma_commit(smem_u32(&bars->empty[stage]));           // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        if (tile.k_end <= tile.k_begin) {
+          // empty contraction (an expert with no rows): nothing was accumulated; the epilogue writes zeros
+        }
+        umma_commit(smem_u32(&bars->acc_full[buf]));
+      }
+    }
+  } else {
+    // ===== epilogue: TMEM -> registers -> global =====
+    const int quarter = warp & 3;                               // TMEM lanes 32*quarter .. +31 belong to this warp
+    uint32_t local = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x, ++local) {
+      const Tile tile = decode_tile(p, t, false);
+      const uint32_t buf = local & 1u;
+      const uint32_t use = local >> 1;
+      const bool got = mbar_wait(smem_u32(&bars->acc_full[buf]), use & 1u, abort_flag, p.status);
+      if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }        // keep the warp converged for tcgen05.ld
+      tc_fence_after();
+      const int row = tile.m0 + quarter * 32 + lane;
+      const bool row_ok = row < tile.m_limit;
+      OutT* row_ptr = static_cast<OutT*>(p.C) + tile.c_off + static_cast<int64_t>(row) * p.ldc;
+      const uint32_t taddr = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(quarter * 32) << 16);
+      const bool empty_k = tile.k_end <= tile.k_begin;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t acc[32];
+        tmem_ld32(taddr + c * 32, acc);
+        tmem_ld_wait();
+        if (c == BN / 32 - 1) {
+          // every value of this accumulator is now in registers: hand the buffer back to the MMA warp
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+        }
+        if (empty_k) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = 0u;
+        }
+        const int col0 = tile.n0 + c * 32;
+        if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, p.accumulate != 0);
+      }
+    }
+  }
+
+  // ===== teardown =====
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D BF16 tensor map over a row-major [rows, cols] matrix with pitch ld (elements); box = {box_cols, box_rows}.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_MN, bool B_MN, typename OutT>
+cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid, cudaStream_t st) {
+  auto kern = gemm_kernel<A_MN, B_MN, OutT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, kp);
+  return cudaGetLastError();
+}
+
+template <typename OutT>
+cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid,
+                          cudaStream_t st) {
+  if (!a.a_mn_major && !a.b_mn_major) return launch_t<false, false, OutT>(tmA, tmB, kp, grid, st);
+  if (!a.a_mn_major && a.b_mn_major) return launch_t<false, true, OutT>(tmA, tmB, kp, grid, st);
+  if (a.a_mn_major && a.b_mn_major) return launch_t<true, true, OutT>(tmA, tmB, kp, grid, st);
+  return launch_t<true, false, OutT>(tmA, tmB, kp, grid, st);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
+  if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
+  KParams kp{};
+  kp.C = a.C;
+  kp.Mo = a.Mo;
+  kp.No = a.No;
+  kp.Kc = a.Kc;
+  kp.ldc = a.ldc;
+  kp.c_dtype = a.c_dtype;
+  kp.accumulate = a.accumulate ? 1 : 0;
+  kp.group_mode = a.group_mode;
+  kp.G = a.G;
+  kp.offs = a.group_offsets;
+  kp.c_group_stride = a.c_group_stride;
+  kp.status = a.status_word;
+  const int64_t a_rows_total = a.group_mode == 1 ? a.rows_padded : a.Mo;   // rows of A (and of C) in mode 1
+  kp.tiles_m = static_cast<int>((a_rows_total + BM - 1) / BM);
+  kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
+  kp.num_tiles = kp.tiles_m * kp.tiles_n * (a.group_mode == 2 ? a.G : 1);
+  if (a.group_mode == 1) kp.Mo = a.rows_padded;
+  if (kp.num_tiles <= 0) return cudaSuccess;
+
+  // Tensor maps. K-major operand: matrix [rows, contraction]; MN-major operand: matrix [contraction, rows].
+  const int64_t contraction_rows = a.group_mode == 2 ? a.rows_padded : a.Kc;
+  CUtensorMap tmA, tmB;
+  bool ok;
+  if (a.a_mn_major) ok = make_map(&tmA, a.A, contraction_rows, a.Mo, a.lda, 64, BK);
+  else ok = make_map(&tmA, a.A, a_rows_total, a.Kc, a.lda, BK, BM);
+  if (!ok) return cudaErrorInvalidValue;
+  const int64_t groups_b = a.group_mode == 1 ? a.G : 1;
+  if (a.b_mn_major) {
+    // [groups * Kc, No] (mode 1) or [contraction_rows, No]
+    const int64_t rows = a.group_mode == 1 ? groups_b * a.Kc : contraction_rows;
+    ok = make_map(&tmB, a.B, rows, a.No, a.ldb, 64, BK);
+    kp.b_group_rows = a.Kc;
+  } else {
+    ok = make_map(&tmB, a.B, groups_b * a.No, a.Kc, a.ldb, BK, BN);
+    kp.b_group_rows = a.No;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+
+  const int grid = kp.num_tiles < kNumSMs ? kp.num_tiles : kNumSMs;
+  if (a.c_dtype == QF_DT_F32) return launch_majors<float>(a, tmA, tmB, kp, grid, st);
+  return launch_majors<__nv_bfloat16>(a, tmA, tmB, kp, grid, st);
+}
+
+}  // namespace qf

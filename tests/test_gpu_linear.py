@@ -1,0 +1,174 @@
+"""GPU parity of the quantization-aware linear layer (forward and straight-through backward)
+against the CPU oracle, through the C ABI. Tolerance (stated by the benchmark spec): max|diff| <= 1e-2 *
+rms(reference), judged on FP32 outputs; BF16 outputs must be the BF16 rounding of the same
+accumulator up to one unit in the last place."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39223_b200 import api, synth
+from util import bits_to_f32, torch_to_bits
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def _rms(a):
+    return float(np.sqrt(np.mean(np.square(a.astype(np.float64)))))
+
+
+def _close(got, ref, what):
+    got = got.detach().float().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    err = float(np.abs(got.astype(np.float64) - ref.astype(np.float64)).max())
+    bound = TOL * _rms(ref)
+    assert err <= bound, f"{what}: max|diff| {err:.3e} > {bound:.3e}"
+
+
+def _bf16_is_rounding_of(bf, f32, what):
+    a = bf.float().cpu().numpy()
+    b = f32.to(torch.bfloat16).float().cpu().numpy()
+    ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(b), 1e-30))) - 7)
+    assert np.all(np.abs(a - b) <= ulp * 1.0001), what
+
+
+COMBOS = [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NVFP4, api.FMT_NONE), (api.FMT_NVFP4, api.FMT_NVFP4),
+          (api.FMT_Q4_K, api.FMT_NONE), (api.FMT_NONE, api.FMT_NONE), (api.FMT_MXFP4, api.FMT_NONE)]
+
+
+@pytest.mark.parametrize("wq,aq", COMBOS)
+@pytest.mark.parametrize("M,N,K", [(128, 256, 256), (200, 264, 768), (1, 8, 256), (333, 520, 1024)])
+def test_small_complete_shapes(wq, aq, M, N, K):
+    c = synth.linear_case(M, N, K, seed=M + N, outlier_channels=2)
+    xb, wb, dyb = (torch_to_bits(t) for t in (c.X, c.W, c.dY))
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    y_ref = oracle.fq_linear_fwd(xb, wb, wq, aq)
+    dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, wq, aq)
+    y32 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32)
+    dx32, dw32 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    _close(y32, y_ref, "Y")
+    _close(dx32, dx_ref, "dX")
+    _close(dw32, dw_ref, "dW")
+    y16 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.bfloat16)
+    dx16, dw16 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.bfloat16, dw_dtype=torch.bfloat16)
+    _bf16_is_rounding_of(y16, y32, "Y bf16")
+    _bf16_is_rounding_of(dx16, dx32, "dX bf16")
+    _bf16_is_rounding_of(dw16, dw32, "dW bf16")
+
+
+def test_one_hot_rows_read_out_quantized_weights_exactly():
+    K, N = 256, 264
+    W = synth.randn_bf16((N, K), 0.02, 1).cuda()
+    eye = torch.eye(K, dtype=torch.bfloat16, device="cuda")
+    y = api.qf_fq_linear_fwd(eye, W, api.FMT_NVFP4, api.FMT_NVFP4, y_dtype=torch.float32)
+    w_hat = api.qf_qdq(api.FMT_NVFP4, W)["out"]
+    assert torch.equal(y, w_hat.float().T)
+
+
+def test_accumulate_dw_and_partial_requests():
+    c = synth.linear_case(256, 256, 512, seed=3)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    dx, dw = api.qf_fq_linear_bwd(dY, X, W, api.FMT_MXFP4, api.FMT_MXFP4)
+    acc = dw.clone()
+    api.qf_fq_linear_bwd(dY, X, W, api.FMT_MXFP4, api.FMT_MXFP4, want_dx=False, dW=acc, flags=api.ACCUMULATE_DW)
+    assert torch.allclose(acc, 2 * dw, rtol=1e-6, atol=0)
+    dx2, none = api.qf_fq_linear_bwd(dY, None, W, api.FMT_MXFP4, api.FMT_MXFP4, want_dw=False)
+    assert none is None and torch.equal(dx2, dx)
+
+
+def test_status_word_is_clean_and_runs_are_deterministic():
+    c = synth.linear_case(512, 512, 512, seed=4)
+    X, W = c.X.cuda(), c.W.cuda()
+    ws = api.workspace(api.OP_LINEAR_FWD, 512, 512, 512)
+    a = api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_MXFP4, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    b = api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_MXFP4, ws=ws)
+    assert torch.equal(a, b)
+
+
+def test_nvfp4_scales_written_back_and_amax_reported():
+    c = synth.linear_case(256, 256, 256, seed=5)
+    X, W = c.X.cuda(), c.W.cuda()
+    wts = torch.zeros(1, device="cuda"); ats = torch.zeros(1, device="cuda"); amax = torch.zeros(1, device="cuda")
+    api.qf_fq_linear_fwd(X, W, api.FMT_NVFP4, api.FMT_NVFP4, w_tscale=wts, a_tscale=ats, a_amax_out=amax)
+    assert wts.item() == np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.W))["tensor_scale"])
+    assert ats.item() == np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.X))["tensor_scale"])
+    assert amax.item() == c.X.abs().max().item()
+    # a supplied (tied / running) scale is honoured
+    given = torch.tensor([float(wts.item()) * 2], device="cuda")
+    y = api.qf_fq_linear_fwd(X, W, api.FMT_NVFP4, api.FMT_NONE, w_tscale=given, flags=api.W_TSCALE_GIVEN, y_dtype=torch.float32)
+    ref = oracle.fq_linear_fwd(torch_to_bits(c.X), torch_to_bits(c.W), api.FMT_NVFP4, api.FMT_NONE, w_tscale=float(given.item()))
+    _close(y, ref, "Y with given scale")
+
+
+def test_full_size_mxfp4_linear_sampled_rows():
+    """The benchmark's workload and launch configuration: X 8192x4096, W 12288x4096, dY 8192x12288,
+    MXFP4 weights and activations. The oracle recomputes sampled output rows with full contractions."""
+    M, N, K = 8192, 12288, 4096
+    c = synth.linear_case(M, N, K, seed=0, device="cuda")
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    y = api.qf_fq_linear_fwd(c.X, c.W, api.FMT_MXFP4, api.FMT_MXFP4, y_dtype=torch.float32, ws=ws)
+    dx, dw = api.qf_fq_linear_bwd(c.dY, c.X, c.W, api.FMT_MXFP4, api.FMT_MXFP4, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(M, 24, replace=False)); rows[0] = 0; rows[-1] = M - 1
+    xb, wb = torch_to_bits(c.X), torch_to_bits(c.W)
+    w_hat = oracle.qdq_out(api.FMT_MXFP4, wb)
+    x_hat = oracle.qdq_out(api.FMT_MXFP4, xb)
+    _close(y[rows], oracle.matmul_fwd(x_hat[rows], w_hat), "Y rows")
+    dyb = torch_to_bits(c.dY)
+    _close(dx[rows], oracle.matmul_dgrad(dyb[rows], w_hat), "dX rows")
+    n_idx = np.sort(rng.choice(N, 16, replace=False)); n_idx[0] = 0; n_idx[-1] = N - 1
+    _close(dw[n_idx], oracle.matmul_wgrad(dyb, x_hat, n_idx), "dW rows")
+
+
+def _grouped_reference(Xp, W, offs, wq, aq, dYp=None):
+    G = W.shape[0]
+    ys, dxs, dws = [], [], []
+    for g in range(G):
+        a, b = int(offs[g]), int(offs[g + 1])
+        xb, wb = torch_to_bits(Xp[a:b]), torch_to_bits(W[g])
+        if b > a:
+            ys.append(oracle.fq_linear_fwd(xb, wb, wq, aq))
+        if dYp is not None:
+            dyb = torch_to_bits(dYp[a:b])
+            if b > a:
+                dx, dw = oracle.fq_linear_bwd(dyb, xb, wb, wq, aq)
+            else:
+                dx, dw = np.zeros((0, W.shape[2]), np.float32), np.zeros(W.shape[1:], np.float32)
+            dxs.append(dx); dws.append(dw)
+    return np.concatenate(ys), (np.concatenate(dxs) if dxs else None), (np.stack(dws) if dws else None)
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NONE, api.FMT_NONE)])
+def test_grouped_small_with_ragged_and_empty_experts(wq, aq):
+    tokens, E, top_k, H, F = 96, 6, 2, 256, 264
+    r = synth.moe_routing(tokens, E, top_k, seed=1)
+    # force one empty expert by giving it no segment
+    X = synth.randn_bf16((tokens, H), 1.0, 2)
+    Xp = synth.gather_rows(X, r.token_of_row)
+    W = synth.randn_bf16((E, F, H), 0.02, 3)
+    dYp = synth.randn_bf16((Xp.shape[0], F), 1e-3, 4)
+    dYp[r.token_of_row < 0] = 0
+    offs = r.group_offsets
+    y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, wq, aq, dYp)
+    offs_d = offs.cuda()
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs_d, wq, aq, y_dtype=torch.float32)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs_d, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    _close(y, y_ref, "grouped Y")
+    _close(dx, dx_ref, "grouped dX")
+    _close(dw, dw_ref, "grouped dW")
+
+
+def test_grouped_empty_expert_gives_zero_dw():
+    E, H, F = 3, 256, 256
+    offs = torch.tensor([0, 128, 128, 256], dtype=torch.int32)        # expert 1 has no rows
+    Xp = synth.randn_bf16((256, H), 1.0, 5)
+    W = synth.randn_bf16((E, F, H), 0.02, 6)
+    dYp = synth.randn_bf16((256, F), 1e-3, 7)
+    y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, api.FMT_MXFP4, api.FMT_MXFP4, dYp)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_MXFP4, api.FMT_MXFP4,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32)
+    assert torch.count_nonzero(dw[1]) == 0
+    _close(dw, dw_ref, "grouped dW")
+    _close(dx, dx_ref, "grouped dX")

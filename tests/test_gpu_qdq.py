@@ -1,0 +1,150 @@
+"""GPU parity: the CUDA quantize-dequantize kernels against the CPU oracle, bit for bit, through
+the C ABI. Codes, scales, tensor scale and dequantized BF16 values must all be identical."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39223_b200 import api, synth
+from util import bits_to_f32, bits_to_torch, f32_to_bits, torch_to_bits
+
+pytestmark = pytest.mark.gpu
+FMTS = [(api.FMT_NVFP4, "nvfp4"), (api.FMT_MXFP4, "mxfp4"), (api.FMT_Q4_K, "q4_k")]
+
+
+def _compare(fmt, xbits, tensor_scale=None):
+    x = bits_to_torch(xbits, "cuda")
+    ts = None if tensor_scale is None else torch.tensor([tensor_scale], dtype=torch.float32, device="cuda")
+    g = api.qf_qdq(fmt, x, tensor_scale=ts)
+    torch.cuda.synchronize()
+    o = oracle.qdq(fmt, xbits, tensor_scale)
+    np.testing.assert_array_equal(torch_to_bits(g["out"]), o["out"])
+    np.testing.assert_array_equal(g["codes"].cpu().numpy(), o["codes"])
+    np.testing.assert_array_equal(g["scales"].cpu().numpy(), o["scales"])
+    if fmt == api.FMT_NVFP4:
+        assert np.float32(g["tensor_scale"].item()).tobytes() == np.float32(o["tensor_scale"]).tobytes()
+    # the inverse half alone reproduces the same tensor from the emitted codes and metadata
+    d = api.qf_dequant(fmt, g["codes"], g["scales"], g["tensor_scale"], *xbits.shape)
+    np.testing.assert_array_equal(torch_to_bits(d), o["out"])
+    return g, o
+
+
+def test_hardware_conversions_match_oracle_encoders():
+    rng = np.random.default_rng(0)
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 0.5, 1, 1.5, 2, 3, 4], np.float32)
+    e4 = np.array([oracle.e4m3_value(c) for c in range(0x7F)], np.float32)
+    e4mid = (e4[:-1] + e4[1:]) / 2
+    v = np.concatenate([rng.uniform(-8, 8, 200000), rng.normal(0, 1, 100000), np.exp(rng.uniform(np.log(1e-5), np.log(600), 100000)),
+                        mids, e4, e4mid, np.array([0.0, 1e-30, 1e9, 448, 449, 464, 465, 480, 2.0 ** -10, 2.0 ** -9])]).astype(np.float32)
+    v = np.concatenate([v, -v, np.nextafter(v, np.float32(np.inf)), np.nextafter(v, np.float32(-np.inf))])
+    e2m1, e4m3 = api.qf_selftest_cvt(torch.from_numpy(v).cuda())
+    want2 = np.array([oracle.e2m1_encode(x) for x in v], np.uint8)
+    want4 = np.array([oracle.e4m3_encode(abs(x)) for x in v], np.uint8)
+    np.testing.assert_array_equal(e2m1.cpu().numpy(), want2)
+    np.testing.assert_array_equal(e4m3.cpu().numpy(), want4)
+
+
+@pytest.mark.parametrize("fmt,name", FMTS)
+@pytest.mark.parametrize("shape", [(1, 256), (3, 512), (37, 768), (129, 2304), (5, 8192)])
+def test_random_weights_small_and_ragged(fmt, name, shape):
+    w = synth.weight_with_outliers(*shape, seed=shape[0])
+    _compare(fmt, torch_to_bits(w))
+
+
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_wide_dynamic_range_blocks(fmt, name):
+    rng = np.random.default_rng(5)
+    rows, cols = 64, 1024
+    x = rng.normal(0, 1, (rows, cols)) * np.exp2(rng.integers(-30, 30, (rows, cols // 16))).repeat(16, axis=1)
+    x[rng.random((rows, cols)) < 0.05] = 0.0
+    x[:, 256:512] = 0.0                                   # whole zero blocks / super-blocks
+    x[3, 512:544] = -0.0
+    _compare(fmt, f32_to_bits(x))
+
+
+def test_nvfp4_exact_ties_and_given_scale():
+    # with s_t = 2^-10 and a block maximum of 2.625 the block scale is 448 and S = 7/16, so these
+    # inputs sit exactly on the rounding midpoints 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5 (times S)
+    ties = np.array([0.109375, 0.328125, 0.546875, 0.765625, 1.09375, 1.53125, 2.1875], np.float32)
+    x = np.zeros((4, 64), np.float32)
+    x[0, :7] = ties; x[0, 15] = 2.625
+    x[1, :7] = -ties; x[1, 15] = -2.625
+    x[2, 16:23] = ties; x[2, 31] = 2.625; x[2, 0] = 1e-6      # first block underflows to scale 0
+    x[3, :] = 2.625
+    g, o = _compare(api.FMT_NVFP4, f32_to_bits(x), tensor_scale=2.0 ** -10)
+    assert list(bits_to_f32(o["out"])[0, :7] / 0.4375) == [0, 1, 1, 2, 2, 4, 4]
+    _compare(api.FMT_NVFP4, f32_to_bits(x))               # derived scale: the same 2^-10
+    _compare(api.FMT_NVFP4, f32_to_bits(x), tensor_scale=3.1e-4)   # a tied / running scale that clips blocks
+
+
+def test_nvfp4_degenerate_tensors():
+    _compare(api.FMT_NVFP4, np.zeros((2, 64), np.uint16))
+    _compare(api.FMT_NVFP4, f32_to_bits(np.full((2, 64), 0.3125)))
+    x = np.full((2, 64), 1e-4, np.float32); x[0, 0] = 3e4
+    _compare(api.FMT_NVFP4, f32_to_bits(x))
+    sub = np.full((2, 64), 2.0 ** -130, np.float32)       # BF16 subnormals everywhere
+    _compare(api.FMT_NVFP4, f32_to_bits(sub))
+
+
+def test_mxfp4_ties_clipping_subnormals_extremes():
+    x = np.zeros((4, 128), np.float32)
+    x[0, :8] = [7, 5, 2.5, 3.5, 0.25, 0.75, 1.25, 1.75]
+    x[0, 32:40] = [-7, -5, -2.5, -3.5, -0.25, -0.75, -1.25, -1.75]
+    x[0, 64:66] = [3.90625, 1]
+    x[1, :32] = 2.0 ** -133
+    x[1, 32:64] = np.linspace(1, 127, 32) * 2.0 ** -133
+    x[1, 64] = 3.0e38; x[1, 65] = 1e30
+    x[1, 96] = 2.0 ** -126; x[1, 97] = 1.5 * 2.0 ** -126
+    x[2, :] = 0.02001953125
+    x[3, 5] = -0.0
+    _compare(api.FMT_MXFP4, f32_to_bits(x))
+
+
+def test_q4k_worked_and_degenerate():
+    x = np.zeros((3, 512), np.float32)
+    x[0, 0:32] = 0.5; x[0, 32:64] = -0.5
+    for b in range(8):
+        x[1, b * 32:(b + 1) * 32] = (b + 1) / 8 * (-1 + 0.125 * (np.arange(32) % 16))
+    x[2, :256] = 0.75
+    x[2, 256:] = -np.abs(np.random.default_rng(1).normal(0, 1, 256))
+    g, o = _compare(api.FMT_Q4_K, f32_to_bits(x))
+    tiny = np.full((1, 256), 2.0 ** -40, np.float32)      # d underflows FP16 -> everything collapses to -em
+    _compare(api.FMT_Q4_K, f32_to_bits(tiny))
+
+
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_two_runs_are_bitwise_identical(fmt, name):
+    x = synth.weight_with_outliers(256, 4096, seed=9, device="cuda")
+    a = api.qf_qdq(fmt, x)
+    b = api.qf_qdq(fmt, x)
+    for k in ("out", "codes", "scales"):
+        assert torch.equal(a[k], b[k])
+
+
+def test_optional_outputs_and_empty_tensor():
+    x = synth.weight_with_outliers(16, 512, seed=2, device="cuda")
+    full = api.qf_qdq(api.FMT_MXFP4, x)
+    only_out = api.qf_qdq(api.FMT_MXFP4, x, want_codes=False, want_scales=False)
+    only_codes = api.qf_qdq(api.FMT_MXFP4, x, want_out=False)
+    assert only_out["codes"] is None and torch.equal(only_out["out"], full["out"])
+    assert only_codes["out"] is None and torch.equal(only_codes["codes"], full["codes"])
+    e = api.qf_qdq(api.FMT_NVFP4, torch.empty((0, 64), dtype=torch.bfloat16, device="cuda"))
+    assert e["tensor_scale"].item() == 1.0
+    assert api.qf_amax(x).item() == x.abs().max().item()
+
+
+def test_full_size_nvfp4_weight_2048():
+    w = synth.nvfp4_weight_2048()
+    _compare(api.FMT_NVFP4, torch_to_bits(w))
+
+
+@pytest.mark.parametrize("name", ["k_proj", "down_proj"])
+def test_full_size_q4k_decoder_matrices(name):
+    # one narrow and one wide matrix of the 32-layer dense decoder, complete and bit-exact
+    w = synth.dense_decoder_weight(3, name)
+    _compare(api.FMT_Q4_K, torch_to_bits(w))
+
+
+def test_full_size_mxfp4_activation():
+    x = synth.activations_with_outlier_channels(8192, 4096, seed=0)
+    _compare(api.FMT_MXFP4, torch_to_bits(x))
