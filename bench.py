@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the fake-quantization hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the whole path over one batch: the quantization-aware linear layer with
+MXFP4 weights and activations, forward plus straight-through backward (dX and dW), on
+X [8192,4096], W [12288,4096], dY [8192,12288] — i.e. two quantize-dequantize passes over W and X
+(forward, and again in the backward, since the fake-quantized copies are transient) and three BF16
+tensor-core matmuls. Prints ONE JSON line (rank 0). Multi-GPU runs are independent replicas of
+the same workload (the path has no exchange step): weak scaling, no data-path collective.
+
+`--impl reference` times the CPU oracle (the only other place this file may execute `oracle/`).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+M, N, K = 8192, 12288, 4096
+WORKLOAD = "mxfp4_w4a4_linear_fwd_bwd_8192x4096x12288"
+FLOP_PER_GEMM = 2.0 * M * N * K
+FLOP_PER_STEP = 3.0 * FLOP_PER_GEMM
+SECTIONS = ("roofline", "qdq", "e2e", "cpu")
+
+
+def _set_shape(spec: str):
+    """--shape M,N,K: a smaller case of the same workload, for profiler captures only."""
+    global M, N, K, WORKLOAD, FLOP_PER_GEMM, FLOP_PER_STEP
+    M, N, K = (int(v) for v in spec.split(","))
+    WORKLOAD = f"mxfp4_w4a4_linear_fwd_bwd_{M}x{K}x{N}"
+    FLOP_PER_GEMM = 2.0 * M * N * K
+    FLOP_PER_STEP = 3.0 * FLOP_PER_GEMM
+KERNELS_PER_STEP = 7          # fwd: qdq(W), qdq(X), gemm; bwd: qdq(W), gemm, qdq(X), gemm
+
+
+def _peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def _physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# -------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded slice of the same workload
+# -------------------------------------------------------------------------------------------------
+
+def _oracle_slice(m_rows: int, n_rows: int, seed: int = 0):
+    """fwd + dX + dW of the MXFP4 W4A4 layer on an [m_rows, K] x [n_rows, K] slice; returns (seconds, flop)."""
+    import numpy as np
+    import oracle
+    from paper_2609_39223_b200 import synth
+    c = synth.linear_case(m_rows, n_rows, K, seed=seed)
+    to_bits = lambda t: t.contiguous().view(__import__("torch").int16).numpy().view(np.uint16)
+    xb, wb, dyb = to_bits(c.X), to_bits(c.W), to_bits(c.dY)
+    t0 = time.perf_counter()
+    oracle.fq_linear_fwd(xb, wb, oracle.FMT_MXFP4, oracle.FMT_MXFP4)
+    oracle.fq_linear_bwd(dyb, xb, wb, oracle.FMT_MXFP4, oracle.FMT_MXFP4)
+    dt = time.perf_counter() - t0
+    return dt, 3.0 * 2.0 * m_rows * n_rows * K
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cores = oracle.num_threads()
+    n_rows = 512
+    # size the slice so that steps+warmup stay within about two minutes
+    dt, fl = _oracle_slice(64, n_rows)
+    rate = fl / dt
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    m_rows = int(max(8, min(512, (rate * budget) / (6.0 * n_rows * K))))
+    for _ in range(args.warmup):
+        _oracle_slice(m_rows, n_rows)
+    t_total, fl_total = 0.0, 0.0
+    for i in range(args.steps):
+        dt, fl = _oracle_slice(m_rows, n_rows, seed=i)
+        t_total += dt
+        fl_total += fl
+    value = fl_total / t_total / 1e12
+    sample = f"fwd+dX+dW on a [{m_rows},{K}] x [{n_rows},{K}] slice per step (QDQ of both slices included)"
+    print(json.dumps({
+        "impl": "reference", "metric": "fake-quant linear fwd+bwd TFLOPS", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# -------------------------------------------------------------------------------------------------
+# our arm
+# -------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_39223_b200 import api, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device — the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    api.lib()
+    peaks = _peaks()
+    fmt = api.FMT_MXFP4
+
+    case = synth.linear_case(M, N, K, seed=rank, device=dev)
+    X, W, dY = case.X, case.W, case.dY
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K, device=dev)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device=dev)
+    dW = torch.empty((N, K), dtype=torch.float32, device=dev)
+
+    def step():
+        api.qf_fq_linear_fwd(X, W, fmt, fmt, ws=ws, Y=Y)
+        api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, ws=ws, dX=dX, dW=dW)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- headline: K steps, inputs resident in HBM -------------------------------------------------
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(_physical_gpu_index(local_rank)) as clk:
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    status = api.qf_read_status(ws)
+    if status != 0:
+        raise SystemExit(f"bench.py: device-side status {status} ({api.status_string(status)})")
+    value = world * FLOP_PER_STEP * args.steps / (ms * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the tcgen05 matmul), timed alone on the same operands ------
+    # The three matmuls of a step are launched here on the already fake-quantized operands (format NONE
+    # skips the quantizers), each launch bracketed by CUDA events on the launching stream.
+    sections = set(args.sections.split(",")) if args.sections else set()
+    achieved, gemm_ms = None, None
+    Xh = api.qf_qdq(fmt, X, want_codes=False, want_scales=False)["out"]
+    Wh = api.qf_qdq(fmt, W, want_codes=False, want_scales=False)["out"]
+    n_rep = max(3, min(args.steps, 20)) if "roofline" in sections else -2
+    evs = []
+
+    def timed(f):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); f(); b.record()
+        evs.append((a, b))
+
+    for it in range(n_rep + 2):
+        if it == 2:
+            evs.clear()
+        timed(lambda: api.qf_fq_linear_fwd(Xh, Wh, 0, 0, ws=ws, Y=Y))
+        timed(lambda: api.qf_fq_linear_bwd(dY, None, Wh, 0, 0, ws=ws, dX=dX, want_dw=False))
+        timed(lambda: api.qf_fq_linear_bwd(dY, Xh, None, 0, 0, ws=ws, dW=dW, want_dx=False))
+    torch.cuda.synchronize()
+    if evs:
+        gemm_ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+        achieved = FLOP_PER_GEMM / (gemm_ms * 1e-3) / 1e12
+    del Xh, Wh
+
+    # ---- QDQ bandwidth per format (memory-bound kernels; reported beside the headline) ---------------
+    qdq = {}
+    if rank == 0 and "qdq" in sections:
+        Wq = synth.randn_bf16((14336, 4096 * 2), 0.02, 7, device=dev)          # 235 MB in, larger than L2
+        out = torch.empty_like(Wq)
+        codes = torch.empty((Wq.shape[0], Wq.shape[1] // 2), dtype=torch.uint8, device=dev)
+        wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
+        for name, f in (("nvfp4", api.FMT_NVFP4), ("mxfp4", api.FMT_MXFP4), ("q4_k", api.FMT_Q4_K)):
+            sc = torch.empty(api.scales_shape(f, *Wq.shape), dtype=torch.uint8, device=dev)
+            for _ in range(3):
+                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(10):
+                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq)
+            b.record(); torch.cuda.synchronize()
+            bytes_per_elem = 2 + 2 + 0.5 + (1 / 32 if f == api.FMT_MXFP4 else 1 / 16)
+            gbs = Wq.numel() * bytes_per_elem / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
+            qdq[name] = {"gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                         "bytes_per_elem": bytes_per_elem}
+        del Wq, out, codes
+
+    # ---- end to end: host buffers, H2D of the inputs and D2H of the results inside the timed region ---
+    e2e = None
+    if "e2e" in sections:
+        hX, hW, hdY = (t.cpu().pin_memory() for t in (X, W, dY))
+        hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        hdX = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+        hdW = torch.empty((N, K), dtype=torch.float32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in (hX, hW, hdY))
+        d2h = sum(t.numel() * t.element_size() for t in (hY, hdX, hdW))
+
+        def e2e_step():
+            X.copy_(hX, non_blocking=True); W.copy_(hW, non_blocking=True); dY.copy_(hdY, non_blocking=True)
+            step()
+            hY.copy_(Y, non_blocking=True); hdX.copy_(dX, non_blocking=True); hdW.copy_(dW, non_blocking=True)
+
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * FLOP_PER_STEP * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    # ---- CPU baseline: the oracle on a bounded slice, rank 0 of a 1-GPU run only -----------------------
+    cpu = None
+    if rank == 0 and world == 1 and "cpu" in sections:
+        import oracle
+        n_rows = 2048
+        dt, fl = _oracle_slice(128, n_rows)                      # calibrate, then aim for about 15 s of CPU work
+        m_rows = int(max(128, min(M, 15.0 * (fl / dt) / (6.0 * n_rows * K)))) // 128 * 128
+        dt, fl = _oracle_slice(m_rows, n_rows)
+        cpu = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"fwd+dX+dW on a [{m_rows},{K}] x [{n_rows},{K}] slice of the workload, QDQ of both slices "
+                         f"included, {dt:.1f} s"}
+
+    if rank == 0:
+        clocks = clk.summary()
+        peak = peaks["bf16_burst"]
+        line = {
+            "metric": "fake-quant linear fwd+bwd TFLOPS", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "wq_fmt": "mxfp4", "aq_fmt": "mxfp4", "M": M, "N": N, "K": K,
+                       "outputs": "Y bf16, dX bf16, dW f32", "parallelism": f"replicas x{world}",
+                       "l2": "inputs (369 MB) larger than L2; no flush"},
+            "clocks": clocks,
+            "e2e": e2e,
+            "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "roofline": {"bound": "tensor", "kernel": "gemm_kernel (tcgen05 BF16, 128x256x64 tiles)", "achieved": achieved,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                         "peak_source": f"{peaks['source']} cuBLAS bf16 burst", "ms_per_launch": gemm_ms,
+                         "frac_of_sustained": achieved / peaks["bf16_sustained"] if achieved else None,
+                         "frac_of_2250_datasheet": achieved / 2250.0 if achieved else None,
+                         "step_frac_of_burst": value / world / peak},
+            "cpu_baseline": cpu,
+            "qdq_gbs": qdq,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sections", default=",".join(SECTIONS),
+                    help="extra measurements beside the headline: roofline,qdq,e2e,cpu (empty string: none)")
+    ap.add_argument("--shape", default=None, help="M,N,K of a smaller case (profiler captures only)")
+    args = ap.parse_args()
+    if args.shape:
+        _set_shape(args.shape)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
