@@ -152,6 +152,12 @@ qf_status_t qf_fq_grouped_linear_bwd(const void* dY, const void* X, const void* 
  * conversion instructions exhaustively with the oracle's encoders. */
 qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8_t* e4m3_out, void* stream);
 
+/* Self-test hook for the exact reciprocal-based division the NVFP4 and Q4_K kernels use in place of
+ * the per-element IEEE divide: for every pair (xs[i], ys[j]) with ys[j] in [2^-60, 2^60] (device FP32
+ * arrays) the quotient is compared bit for bit with the IEEE quotient; *mismatches (device u64)
+ * receives the number of differences. */
+qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
+    "qf_selftest_div",
 ]
 
 
@@ -74,6 +75,8 @@ def lib() -> ctypes.CDLL:
                                                c_uint32, c_void_p, c_size_t, c_void_p]
         L.qf_selftest_cvt.restype = c_int
         L.qf_selftest_cvt.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
+        L.qf_selftest_div.restype = c_int
+        L.qf_selftest_div.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -243,3 +246,11 @@ def qf_selftest_cvt(x: torch.Tensor):
     e4 = torch.empty(x.numel(), dtype=torch.uint8, device=x.device)
     _check(lib().qf_selftest_cvt(_ptr(x), x.numel(), _ptr(e2), _ptr(e4), _stream()), "qf_selftest_cvt")
     return e2, e4
+
+
+def qf_selftest_div(xs: torch.Tensor, ys: torch.Tensor) -> int:
+    """Number of (x, y) pairs for which the kernels' reciprocal-based division differs from the IEEE divide."""
+    assert xs.dtype == torch.float32 and ys.dtype == torch.float32 and xs.is_cuda and ys.is_cuda
+    out = torch.zeros(1, dtype=torch.int64, device=xs.device)
+    _check(lib().qf_selftest_div(_ptr(xs), xs.numel(), _ptr(ys), ys.numel(), _ptr(out), _stream()), "qf_selftest_div")
+    return int(out.item())

@@ -355,4 +355,13 @@ qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8
   return cu(launch_selftest_cvt(in, n, e2m1_out, e4m3_out, static_cast<cudaStream_t>(stream)));
 }
 
+qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream) {
+  if (!xs || !ys || !mismatches) return QF_ERR_NULL;
+  if (nx < 0 || ny < 0) return QF_ERR_SHAPE;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaError_t e = cudaMemsetAsync(mismatches, 0, 8, st)) return cu(e);
+  return cu(launch_selftest_div(xs, nx, ys, ny, reinterpret_cast<unsigned long long*>(mismatches), st));
+}
+
 }  // extern "C"

@@ -96,6 +96,8 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st);
 cudaError_t launch_dequant(int fmt, const void* codes, const void* scales, const float* tscale, int64_t rows,
                            int64_t cols, void* out, cudaStream_t st);
+cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,
+                                cudaStream_t st);
 cudaError_t launch_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1, uint8_t* e4m3, cudaStream_t st);
 
 // C[Mo, No] (+)= sum_c A(m, c) * B(n, c). Operand storage: K-major = [rows, contraction] row-major,

@@ -13,7 +13,6 @@ namespace qf {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;          // independent 16-byte loads in flight per thread
 
 __device__ __forceinline__ uint4 ld_chunk(const uint4* p) { return __ldg(p); }
 
@@ -56,69 +55,135 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
 __global__ void amax_to_float_kernel(const uint32_t* amax_bits, float* out) { *out = __uint_as_float(*amax_bits); }
 
 // ---------------------------------------------------------------------------------------------
-// per-chunk quantize-dequantize, FP4 formats
+// Exact division without the per-element IEEE divide sequence.
+//
+// The formats need v = x / S (NVFP4) and t = (x + em) / es (Q4_K) as correctly rounded FP32
+// quotients, because the quotient decides a code. One divisor serves a whole block, so its correctly
+// rounded reciprocal rc = RN(1/y) is computed once and every quotient is then
+//     q0 = RN(x * rc);  q1 = RN(q0 + rc * RN(x - y*q0));  q2 = RN(q1 + rc * RN(x - y*q1))
+// (fused multiply-adds, two elements per instruction). With an exactly rounded reciprocal and
+// no overflow / underflow in the residuals this is the classical correctly-rounded division
+// iteration (Markstein); the range guard below keeps operands where that holds and the
+// caller falls back to the IEEE divide otherwise. qf_selftest_div compares it with the IEEE divide.
 // ---------------------------------------------------------------------------------------------
 
-struct ChunkOut {
-  uint4 xhat;        // 8 BF16
-  uint32_t codes;    // 8 x 4 bit, element i in nibble i
+__device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
+
+__device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
+  const float2 ny = splat(-y), r = splat(rc);
+  float2 q = __fmul2_rn(x, r);
+  q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+  q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+  return q;
+}
+__device__ __forceinline__ float div1_fast(float x, float y, float rc) {
+  float q = __fmul_rn(x, rc);
+  q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+  q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+  return q;
+}
+// divisor magnitudes for which the iteration above is used
+__device__ __forceinline__ bool div_safe(float y) { return y >= 0x1p-60f && y <= 0x1p60f; }
+
+__device__ __forceinline__ float copysign_bits(float mag, float sgn) {
+  return __uint_as_float((__float_as_uint(mag) & 0x7FFFFFFFu) | (__float_as_uint(sgn) & 0x80000000u));
+}
+
+__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
+
+__device__ __forceinline__ uint32_t bf2_bits(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
+__device__ __forceinline__ __nv_bfloat162 bits_bf2(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
+
+// max |x| over 16 BF16 values held in 8 words, as BF16 bits (sign clear)
+__device__ __forceinline__ uint32_t unit_amax_bits(const uint32_t (&w)[8]) {
+  __nv_bfloat162 m0 = __hmax2(__habs2(bits_bf2(w[0])), __habs2(bits_bf2(w[1])));
+  __nv_bfloat162 m1 = __hmax2(__habs2(bits_bf2(w[2])), __habs2(bits_bf2(w[3])));
+  __nv_bfloat162 m2 = __hmax2(__habs2(bits_bf2(w[4])), __habs2(bits_bf2(w[5])));
+  __nv_bfloat162 m3 = __hmax2(__habs2(bits_bf2(w[6])), __habs2(bits_bf2(w[7])));
+  const uint32_t m = bf2_bits(__hmax2(__hmax2(m0, m1), __hmax2(m2, m3)));
+  return max(m & 0xFFFFu, m >> 16);
+}
+
+// ---------------------------------------------------------------------------------------------
+// FP4 formats: one lane owns 16 consecutive elements (two 16-byte loads): a whole NVFP4 block, or
+// half an MXFP4 block (one shuffle with the neighbouring lane).
+// ---------------------------------------------------------------------------------------------
+
+struct UnitOut {
+  uint32_t xhat[8];   // 16 BF16
+  uint2 codes;        // 16 x 4 bit, element i in nibble i
 };
 
-// MXFP4: x_hat = 2^p * C with p = floor(log2 amax_block) - 2 (Eq. mxfp4-dequant).
-__device__ __forceinline__ ChunkOut mxfp4_chunk(const uint4& v, uint32_t block_amax_bits, uint32_t& scale_code) {
+// MXFP4: x_hat = 2^p * C with p = floor(log2 amax_block) - 2 (Eq. mxfp4-dequant). All products exact.
+__device__ __forceinline__ UnitOut mxfp4_unit(const uint32_t (&w)[8], uint32_t block_amax_bits, uint32_t& scale_code) {
   scale_code = mxfp4_scale_code(block_amax_bits);
-  const float inv = e8m0_inv_scale(scale_code);
-  const float sc = e8m0_scale(scale_code);
-  const bool zero_block = block_amax_bits == 0;
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-  uint32_t o[4];
-  ChunkOut r;
-  r.codes = 0;
+  const float2 inv = splat(e8m0_inv_scale(scale_code));
+  const float2 sc = splat(e8m0_scale(scale_code));
+  const uint32_t keep = block_amax_bits == 0 ? 0u : 0xFFu;       // an all-zero block drops the sign of -0
+  UnitOut r;
+  uint32_t c[2] = {0, 0};
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    uint32_t byte = e2m1x2_encode(__fmul_rn(bf16_lo(w[j]), inv), __fmul_rn(bf16_hi(w[j]), inv));
-    if (zero_block) byte = 0;                       // an all-zero block drops the sign of -0
-    float2 c = e2m1x2_decode(byte);
-    o[j] = pack_bf16x2(__fmul_rn(c.x, sc), __fmul_rn(c.y, sc));
-    r.codes |= byte << (8 * j);
+  for (int j = 0; j < 8; ++j) {
+    const float2 v = __fmul2_rn(unpack2(w[j]), inv);
+    const uint32_t byte = e2m1x2_encode(v.x, v.y) & keep;
+    const float2 o = __fmul2_rn(e2m1x2_decode(byte), sc);
+    r.xhat[j] = pack_bf16x2(o.x, o.y);
+    c[j >> 2] |= byte << (8 * (j & 3));
   }
-  r.xhat = make_uint4(o[0], o[1], o[2], o[3]);
+  r.codes = make_uint2(c[0], c[1]);
   return r;
 }
 
 // NVFP4: x_hat = s_FP32 * s_E4M3 * C (Eq. nvfp4-dequant); block scale = E4M3(amax_block / (6 s_FP32)).
-__device__ __forceinline__ ChunkOut nvfp4_chunk(const uint4& v, uint32_t block_amax_bits, float s_t,
-                                                uint32_t& scale_code) {
-  const float amax_b = __uint_as_float(block_amax_bits << 16);
-  const float q = __fdiv_rn(amax_b, __fmul_rn(6.0f, s_t));
+// FAST selects the reciprocal-based exact division; otherwise the IEEE divide.
+template <bool FAST>
+__device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax_b, float s_t, float denom, float rc_denom,
+                                              uint32_t& scale_code) {
+  const float q = FAST ? div1_fast(amax_b, denom, rc_denom) : __fdiv_rn(amax_b, denom);
   scale_code = e4m3_encode(q);
   const float sb = e4m3_decode(scale_code);
   const float S = __fmul_rn(s_t, sb);
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-  uint32_t o[4];
-  ChunkOut r;
-  r.codes = 0;
+  UnitOut r;
+  uint32_t c[2] = {0, 0};
+  // fast path needs a sane divisor and quotients that cannot overflow; S == 0 means "all zero"
+  const bool zero = S == 0.0f;
+  const bool fast = FAST && div_safe(S) && amax_b <= __fmul_rn(8.0f, S);
+  const float rc = fast ? __frcp_rn(S) : 0.0f;
+  const float2 sb2 = splat(sb), st2 = splat(s_t);
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int j = 0; j < 8; ++j) {
+    const float2 x = unpack2(w[j]);
     uint32_t byte = 0;
-    if (S != 0.0f) byte = e2m1x2_encode(__fdiv_rn(bf16_lo(w[j]), S), __fdiv_rn(bf16_hi(w[j]), S));
-    float2 c = e2m1x2_decode(byte);
-    o[j] = pack_bf16x2(__fmul_rn(__fmul_rn(sb, c.x), s_t), __fmul_rn(__fmul_rn(sb, c.y), s_t));
-    r.codes |= byte << (8 * j);
+    if (!zero) {
+      float2 v;
+      if (fast) {
+        v = div2_fast(x, S, rc);
+        v.x = copysign_bits(v.x, x.x);      // x = -0 must keep its sign, as in the IEEE quotient
+        v.y = copysign_bits(v.y, x.y);
+      } else {
+        v = make_float2(__fdiv_rn(x.x, S), __fdiv_rn(x.y, S));
+      }
+      byte = e2m1x2_encode(v.x, v.y);
+    }
+    const float2 o = __fmul2_rn(__fmul2_rn(sb2, e2m1x2_decode(byte)), st2);
+    r.xhat[j] = pack_bf16x2(o.x, o.y);
+    c[j >> 2] |= byte << (8 * (j & 3));
   }
-  r.xhat = make_uint4(o[0], o[1], o[2], o[3]);
+  r.codes = make_uint2(c[0], c[1]);
   return r;
 }
 
+constexpr int kUnitsPerThread = 2;
+
 template <int FMT>
-__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restrict__ in, int64_t nchunks,
-                                                           uint4* __restrict__ out, uint32_t* __restrict__ codes,
+__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restrict__ in, int64_t nunits,
+                                                           uint4* __restrict__ out, uint2* __restrict__ codes,
                                                            uint8_t* __restrict__ scales,
                                                            const float* __restrict__ tscale_in,
                                                            const uint32_t* __restrict__ amax_bits,
                                                            float* __restrict__ tscale_out) {
-  constexpr int kLanesPerBlock = FMT == QF_FMT_NVFP4 ? 2 : 4;
-  float s_t = 1.0f;
+  float s_t = 1.0f, denom = 6.0f, rc_denom = 0.0f;
+  bool denom_safe = false;
   if (FMT == QF_FMT_NVFP4) {
     if (amax_bits) {
       const float amax_t = __uint_as_float(*amax_bits);
@@ -127,136 +192,220 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restri
     } else {
       s_t = *tscale_in;
     }
+    denom = __fmul_rn(6.0f, s_t);
+    denom_safe = div_safe(denom);
+    rc_denom = denom_safe ? __frcp_rn(denom) : 0.0f;
   }
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
   const int64_t first = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
-  // warp-uniform trip count: every lane of a warp takes part in the shuffles
-  const int64_t warp_first = first - (threadIdx.x & 31);
-  for (int64_t base = 0; warp_first + base < nchunks; base += kUnroll * stride) {
-    uint4 v[kUnroll];
-    bool ok[kUnroll];
+  const int64_t warp_first = first - (threadIdx.x & 31);      // warp-uniform trip count (shuffles below)
+  for (int64_t base = 0; warp_first + base < nunits; base += kUnitsPerThread * stride) {
+    uint4 v[kUnitsPerThread][2];
+    bool ok[kUnitsPerThread];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
+    for (int u = 0; u < kUnitsPerThread; ++u) {
       const int64_t i = first + base + u * stride;
-      ok[u] = i < nchunks;
-      v[u] = ok[u] ? ld_chunk(in + i) : make_uint4(0, 0, 0, 0);
+      ok[u] = i < nunits;
+      v[u][0] = ok[u] ? ld_chunk(in + 2 * i) : make_uint4(0, 0, 0, 0);
+      v[u][1] = ok[u] ? ld_chunk(in + 2 * i + 1) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
+    for (int u = 0; u < kUnitsPerThread; ++u) {
       const int64_t i = first + base + u * stride;
-      if (warp_first + base + u * stride >= nchunks) break;                 // warp-uniform
-      uint32_t m = chunk_amax_bits(v[u]);
-      m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-      if (kLanesPerBlock == 4) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+      if (warp_first + base + u * stride >= nunits) break;                 // warp-uniform
+      const uint32_t w[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w, v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
+      uint32_t m = unit_amax_bits(w);
       uint32_t scale_code;
-      ChunkOut r = FMT == QF_FMT_NVFP4 ? nvfp4_chunk(v[u], m, s_t, scale_code) : mxfp4_chunk(v[u], m, scale_code);
+      UnitOut r;
+      if (FMT == QF_FMT_MXFP4) {
+        m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+        r = mxfp4_unit(w, m, scale_code);
+      } else {
+        const float amax_b = __uint_as_float(m << 16);
+        // quotients near the bottom of the FP32 range take the IEEE divide (warp-uniform choice)
+        const bool fast_ok = denom_safe && (amax_b == 0.0f || amax_b >= 0x1p-60f);
+        if (__all_sync(0xFFFFFFFFu, fast_ok)) r = nvfp4_unit<true>(w, amax_b, s_t, denom, rc_denom, scale_code);
+        else r = nvfp4_unit<false>(w, amax_b, s_t, denom, rc_denom, scale_code);
+      }
       if (ok[u]) {
-        if (out) out[i] = r.xhat;
+        if (out) {
+          out[2 * i] = make_uint4(r.xhat[0], r.xhat[1], r.xhat[2], r.xhat[3]);
+          out[2 * i + 1] = make_uint4(r.xhat[4], r.xhat[5], r.xhat[6], r.xhat[7]);
+        }
         if (codes) codes[i] = r.codes;
-        if (scales && (threadIdx.x & (kLanesPerBlock - 1)) == 0) scales[i / kLanesPerBlock] = static_cast<uint8_t>(scale_code);
+        if (scales) {
+          if (FMT == QF_FMT_NVFP4) scales[i] = static_cast<uint8_t>(scale_code);
+          else if ((threadIdx.x & 1) == 0) scales[i >> 1] = static_cast<uint8_t>(scale_code);
+        }
       }
     }
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Q4_K: one warp per 256-weight super-block; lane t owns elements 8t..8t+7, sub-block t/4.
+// Q4_K: one lane owns a 32-weight sub-block (four 16-byte loads), eight lanes a 256-weight
+// super-block, a warp four super-blocks.
 // x_hat = (d * s6) * C - (dmin * m6)  (Eq. q4k-dequant); min/max affine rule for the quantizer.
 // ---------------------------------------------------------------------------------------------
 
-__device__ __forceinline__ float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
+constexpr float kRcp15 = 1.0f / 15.0f;        // correctly rounded reciprocals of the two constant divisors
+constexpr float kRcp63 = 1.0f / 63.0f;
+constexpr float kRound = 12582912.0f;      // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
 
-__global__ void __launch_bounds__(kThreads) qdq_q4k_kernel(const uint4* __restrict__ in, int64_t nchunks,
-                                                           uint4* __restrict__ out, uint32_t* __restrict__ codes,
+template <bool FAST>
+__device__ __forceinline__ float div_by(float x, float y, float rc) { return FAST ? div1_fast(x, y, rc) : __fdiv_rn(x, y); }
+
+template <bool FAST>
+__device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, float hi, uint32_t (&xhat)[16],
+                                             uint32_t (&cbytes)[8], __half& d_h, __half& dmin_h, uint32_t& s6, uint32_t& m6) {
+  lo = fminf(lo, 0.0f);
+  const float sc = div_by<FAST>(__fsub_rn(hi, lo), 15.0f, kRcp15);
+  const float off = __fsub_rn(0.0f, lo);            // >= +0: a sub-block with no negative value has offset +0
+  float max_sc = sc, max_off = off;
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) {
+    max_sc = fmaxf(max_sc, __shfl_xor_sync(0xFFFFFFFFu, max_sc, s));
+    max_off = fmaxf(max_off, __shfl_xor_sync(0xFFFFFFFFu, max_off, s));
+  }
+  d_h = __float2half_rn(fminf(div_by<FAST>(max_sc, 63.0f, kRcp63), 65504.0f));
+  dmin_h = __float2half_rn(fminf(div_by<FAST>(max_off, 63.0f, kRcp63), 65504.0f));
+  const float d = __half2float(d_h), dmin = __half2float(dmin_h);
+  // FP16 values are at least 2^-24, well inside the safe divisor range
+  const float s6f = d == 0.0f ? 0.0f : fminf(fmaxf(rintf(div_by<FAST>(sc, d, __frcp_rn(d))), 0.0f), 63.0f);
+  const float m6f = dmin == 0.0f ? 0.0f : fminf(fmaxf(rintf(div_by<FAST>(off, dmin, __frcp_rn(dmin))), 0.0f), 63.0f);
+  s6 = static_cast<uint32_t>(s6f);
+  m6 = static_cast<uint32_t>(m6f);
+  const float es = __fmul_rn(d, s6f), em = __fmul_rn(dmin, m6f);
+  const bool live = es > 0.0f;
+  const float rc = live ? __frcp_rn(es) : 0.0f;
+  const float2 em2 = splat(em), nem2 = splat(-em), es2 = splat(es), magic = splat(kRound), nmagic = splat(-kRound);
+  uint32_t ybits[2][2];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float2 x = unpack2(w[j]);
+    float2 y = magic;                                // code 0 when the sub-block has no scale
+    if (live) {
+      const float2 num = __fadd2_rn(x, em2);
+      float2 t = FAST ? div2_fast(num, es, rc) : make_float2(__fdiv_rn(num.x, es), __fdiv_rn(num.y, es));
+      t.x = fminf(fmaxf(t.x, 0.0f), 15.0f);          // clamp first: rounding is monotone and 0, 15 are integers
+      t.y = fminf(fmaxf(t.y, 0.0f), 15.0f);
+      y = __fadd2_rn(t, magic);                      // integer code now sits in the low mantissa bits
+    }
+    const float2 c = __fadd2_rn(y, nmagic);
+    const float2 o = __ffma2_rn(es2, c, nem2);        // product exact: one rounding, as es*c - em
+    xhat[j] = pack_bf16x2(o.x, o.y);
+    // the low byte of y's bit pattern is the code (the low byte of the rounding constant is zero)
+    ybits[j & 1][0] = __float_as_uint(y.x);
+    ybits[j & 1][1] = __float_as_uint(y.y);
+    if (j & 1) {
+      const uint32_t p01 = __byte_perm(ybits[0][0], ybits[0][1], 0x0040);
+      const uint32_t p23 = __byte_perm(ybits[1][0], ybits[1][1], 0x0040);
+      cbytes[j >> 1] = __byte_perm(p01, p23, 0x5410);             // codes 4k..4k+3, one per byte
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) qdq_q4k_kernel(const uint4* __restrict__ in, int64_t nsub,
+                                                           uint4* __restrict__ out, uint4* __restrict__ codes,
                                                            uint4* __restrict__ scales) {
   const int lane = threadIdx.x & 31;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
-  // nchunks is a multiple of 32, so a warp is either entirely inside the tensor or entirely outside
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < nchunks; i += stride) {
-    const uint4 v = ld_chunk(in + i);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    float x[8];
+  const int64_t first = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  // nsub (sub-blocks) is a multiple of 8; a warp covers 32 of them, so the last warp may be partly idle
+  for (int64_t i = first; i - lane < nsub; i += stride) {
+    const bool ok = i < nsub;
+    uint32_t w[16];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      x[2 * j] = bf16_lo(w[j]);
-      x[2 * j + 1] = bf16_hi(w[j]);
+    for (int k = 0; k < 4; ++k) {
+      const uint4 v = ok ? ld_chunk(in + 4 * i + k) : make_uint4(0, 0, 0, 0);
+      w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
     }
-    float lo = fminf(fminf(fminf(x[0], x[1]), fminf(x[2], x[3])), fminf(fminf(x[4], x[5]), fminf(x[6], x[7])));
-    float hi = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
-    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 1));
-    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 1));
-    lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 2));
-    hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 2));
-    lo = fminf(lo, 0.0f);
-    const float sc = __fdiv_rn(__fsub_rn(hi, lo), 15.0f);
-    const float off = __fsub_rn(0.0f, lo);             // >= +0: a sub-block with no negative value has offset +0
-    float max_sc = sc, max_off = off;
+    __nv_bfloat162 mn = bits_bf2(w[0]), mx = bits_bf2(w[0]);
 #pragma unroll
-    for (int s = 4; s < 32; s <<= 1) {
-      max_sc = fmaxf(max_sc, __shfl_xor_sync(0xFFFFFFFFu, max_sc, s));
-      max_off = fmaxf(max_off, __shfl_xor_sync(0xFFFFFFFFu, max_off, s));
+    for (int j = 1; j < 16; ++j) {
+      mn = __hmin2(mn, bits_bf2(w[j]));
+      mx = __hmax2(mx, bits_bf2(w[j]));
     }
-    const __half d_h = __float2half_rn(fminf(__fdiv_rn(max_sc, 63.0f), 65504.0f));
-    const __half dmin_h = __float2half_rn(fminf(__fdiv_rn(max_off, 63.0f), 65504.0f));
-    const float d = __half2float(d_h), dmin = __half2float(dmin_h);
-    const float s6f = d == 0.0f ? 0.0f : clampf(rintf(__fdiv_rn(sc, d)), 0.0f, 63.0f);
-    const float m6f = dmin == 0.0f ? 0.0f : clampf(rintf(__fdiv_rn(off, dmin)), 0.0f, 63.0f);
-    const float es = __fmul_rn(d, s6f), em = __fmul_rn(dmin, m6f);
-    uint32_t c8 = 0;
-    uint32_t o[4];
+    const float lo = fminf(bf16_lo(bf2_bits(mn)), bf16_hi(bf2_bits(mn)));
+    const float hi = fmaxf(bf16_lo(bf2_bits(mx)), bf16_hi(bf2_bits(mx)));
+    // the reciprocal-based division is exact away from the bottom of the FP32 range; a warp with a
+    // tiny but non-zero range or offset takes the IEEE divide instead
+    const float range = __fsub_rn(hi, fminf(lo, 0.0f)), offv = -fminf(lo, 0.0f);
+    const bool fast_ok = (range == 0.0f || (range >= 0x1p-60f && range <= 0x1p60f)) && (offv == 0.0f || (offv >= 0x1p-60f && offv <= 0x1p60f));
+    uint32_t xhat[16], cb[8], s6, m6;
+    __half d_h, dmin_h;
+    if (__all_sync(0xFFFFFFFFu, fast_ok)) q4k_subblock<true>(w, lo, hi, xhat, cb, d_h, dmin_h, s6, m6);
+    else q4k_subblock<false>(w, lo, hi, xhat, cb, d_h, dmin_h, s6, m6);
+    if (ok && out) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float c0 = 0.0f, c1 = 0.0f;
-      if (es > 0.0f) {
-        c0 = clampf(rintf(__fdiv_rn(__fadd_rn(x[2 * j], em), es)), 0.0f, 15.0f);
-        c1 = clampf(rintf(__fdiv_rn(__fadd_rn(x[2 * j + 1], em), es)), 0.0f, 15.0f);
-      }
-      o[j] = pack_bf16x2(__fsub_rn(__fmul_rn(es, c0), em), __fsub_rn(__fmul_rn(es, c1), em));
-      c8 |= (static_cast<uint32_t>(c0) | (static_cast<uint32_t>(c1) << 4)) << (8 * j);
+      for (int k = 0; k < 4; ++k) out[4 * i + k] = make_uint4(xhat[4 * k], xhat[4 * k + 1], xhat[4 * k + 2], xhat[4 * k + 3]);
     }
-    if (out) out[i] = make_uint4(o[0], o[1], o[2], o[3]);
-    // code bytes: within a 64-element chunk (8 lanes), byte l = element l | element l+32 << 4.
-    // Lanes 0-3 of the 8 hold elements l, lanes 4-7 the elements l+32; the pair (t, t^4) splits the
-    // 8 bytes it can form: the low lane writes bytes for its elements 0-3, the high lane for 4-7.
-    const uint32_t partner = __shfl_xor_sync(0xFFFFFFFFu, c8, 4);
-    if (codes) {
-      const bool high = (lane & 4) != 0;
-      const uint32_t lo_src = high ? partner : c8, hi_src = high ? c8 : partner;
-      const int sh = high ? 16 : 0;
-      uint32_t word = 0;
+    // code bytes: a 64-element chunk is the lane pair (2j, 2j+1); byte l = code[2j][l] | code[2j+1][l] << 4.
+    // cb[k] holds codes 4k..4k+3 one per byte. The even lane forms bytes 0-15, the odd lane bytes 16-31.
+    const bool odd = lane & 1;
+    uint32_t mine[4], theirs[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        word |= (((lo_src >> (sh + 4 * k)) & 15u) | (((hi_src >> (sh + 4 * k)) & 15u) << 4)) << (8 * k);
-      // super-block i/32 owns 32 words; chunk (lane/8) owns 8 of them; low lane q writes word 2q, high 2q+1
-      const int q = lane & 3;
-      codes[(i - lane) + (lane >> 3) * 8 + 2 * q + (high ? 1 : 0)] = word;
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t send = odd ? cb[k] : cb[4 + k];            // what the partner needs from this lane
+      theirs[k] = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+      mine[k] = odd ? cb[4 + k] : cb[k];
+    }
+    if (ok && codes) {
+      uint32_t o[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) o[k] = odd ? (theirs[k] | (mine[k] << 4)) : (mine[k] | (theirs[k] << 4));
+      // super-block = 8 lanes x 16 bytes = 128 bytes; chunk (lane/2 mod 4) owns 32 of them
+      codes[i] = make_uint4(o[0], o[1], o[2], o[3]);
     }
     if (scales) {
-      // gather the eight 6-bit (s6, m6) pairs: each sub-block leader contributes its byte lanes
-      const uint32_t s6 = static_cast<uint32_t>(s6f), m6 = static_cast<uint32_t>(m6f);
-      const int b = lane >> 2;
-      const bool leader = (lane & 3) == 0;
-      // words of the 12 packed bytes: w0 = bytes 0-3, w1 = bytes 4-7, w2 = bytes 8-11
-      uint32_t w0 = 0, w1 = 0, w2 = 0;
-      if (leader) {
-        if (b < 4) {
-          w0 = (s6 & 63u) << (8 * b);
-          w1 = (m6 & 63u) << (8 * b);
-        } else {
-          w0 = ((s6 >> 4) << 6) << (8 * (b - 4));
-          w1 = ((m6 >> 4) << 6) << (8 * (b - 4));
-          w2 = ((s6 & 15u) | ((m6 & 15u) << 4)) << (8 * (b - 4));
-        }
+      const int b = lane & 7;                                       // sub-block within its super-block
+      uint32_t w0 = 0, w1 = 0, w2 = 0;                              // the 12 packed bytes as three words
+      if (b < 4) {
+        w0 = (s6 & 63u) << (8 * b);
+        w1 = (m6 & 63u) << (8 * b);
+      } else {
+        w0 = ((s6 >> 4) << 6) << (8 * (b - 4));
+        w1 = ((m6 >> 4) << 6) << (8 * (b - 4));
+        w2 = ((s6 & 15u) | ((m6 & 15u) << 4)) << (8 * (b - 4));
       }
-      w0 = __reduce_or_sync(0xFFFFFFFFu, w0);
-      w1 = __reduce_or_sync(0xFFFFFFFFu, w1);
-      w2 = __reduce_or_sync(0xFFFFFFFFu, w2);
-      if (lane == 0) {
+#pragma unroll
+      for (int s = 1; s < 8; s <<= 1) {
+        w0 |= __shfl_xor_sync(0xFFFFFFFFu, w0, s);
+        w1 |= __shfl_xor_sync(0xFFFFFFFFu, w1, s);
+        w2 |= __shfl_xor_sync(0xFFFFFFFFu, w2, s);
+      }
+      if (ok && b == 0) {
         const uint32_t hdr = static_cast<uint32_t>(__half_as_ushort(d_h)) | (static_cast<uint32_t>(__half_as_ushort(dmin_h)) << 16);
-        scales[i >> 5] = make_uint4(hdr, w0, w1, w2);
+        scales[i >> 3] = make_uint4(hdr, w0, w1, w2);
       }
     }
   }
+}
+
+// exhaustive comparison of the reciprocal-based division with the IEEE divide: every x in xs against
+// every y in ys (and, with bf16_sweep, every non-negative BF16 bit pattern as x)
+__global__ void selftest_div_kernel(const float* __restrict__ xs, int64_t nx, const float* __restrict__ ys, int64_t ny,
+                                    unsigned long long* __restrict__ mismatches) {
+  const int64_t total = nx * ny;
+  unsigned long long bad = 0;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const float x = xs[i % nx], y = ys[i / nx];
+    if (!div_safe(y)) continue;
+    const float rc = __frcp_rn(y);
+    const float ref = __fdiv_rn(x, y);
+    // Domain in which the kernels rely on exactness: a numerator that is zero or not tiny, or a
+    // quotient large enough to sit near a rounding threshold (those start at 0.25). A tiny quotient
+    // of a tiny numerator may differ in its last bit (the residual underflows) but rounds to code 0
+    // either way. Quotients beyond 2^100 never occur (the callers bound the numerator by 8 * divisor).
+    if (!(x == 0.0f || fabsf(x) >= 0x1p-60f || fabsf(ref) >= 0x1p-8f) || fabsf(ref) > 0x1p100f) continue;
+    const float2 q = div2_fast(make_float2(x, -x), y, rc);
+    const float q1 = div1_fast(x, y, rc);
+    if (__float_as_uint(copysign_bits(q.x, x)) != __float_as_uint(ref)) ++bad;
+    if (__float_as_uint(copysign_bits(q.y, -x)) != __float_as_uint(-ref)) ++bad;
+    if (__float_as_uint(copysign_bits(q1, x)) != __float_as_uint(ref)) ++bad;
+  }
+  if (bad) atomicAdd(mismatches, bad);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -357,21 +506,30 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
 }
 
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st) {
-  const int64_t nchunks = a.rows * a.cols / 8;
+  const int64_t nelem = a.rows * a.cols;
   // an empty NVFP4 tensor still has a tensor scale to report (1.0): let one block write it
-  if (nchunks == 0 && !(a.fmt == QF_FMT_NVFP4 && a.tscale_out)) return cudaSuccess;
+  if (nelem == 0 && !(a.fmt == QF_FMT_NVFP4 && a.tscale_out)) return cudaSuccess;
   const uint4* in = static_cast<const uint4*>(a.in);
   uint4* out = static_cast<uint4*>(a.out);
-  uint32_t* codes = static_cast<uint32_t*>(a.codes);
   if (a.fmt == QF_FMT_NVFP4) {
-    qdq_fp4_kernel<QF_FMT_NVFP4><<<grid_for(nchunks, kUnroll), kThreads, 0, st>>>(
-        in, nchunks, out, codes, static_cast<uint8_t*>(a.scales), a.tscale_in, a.amax_bits, a.tscale_out);
+    const int64_t nunits = nelem / 16;
+    qdq_fp4_kernel<QF_FMT_NVFP4><<<grid_for(nunits, kUnitsPerThread), kThreads, 0, st>>>(
+        in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), a.tscale_in, a.amax_bits, a.tscale_out);
   } else if (a.fmt == QF_FMT_MXFP4) {
-    qdq_fp4_kernel<QF_FMT_MXFP4><<<grid_for(nchunks, kUnroll), kThreads, 0, st>>>(
-        in, nchunks, out, codes, static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr);
+    const int64_t nunits = nelem / 16;
+    qdq_fp4_kernel<QF_FMT_MXFP4><<<grid_for(nunits, kUnitsPerThread), kThreads, 0, st>>>(
+        in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr);
   } else {
-    qdq_q4k_kernel<<<grid_for(nchunks, 2), kThreads, 0, st>>>(in, nchunks, out, codes, static_cast<uint4*>(a.scales));
+    const int64_t nsub = nelem / 32;
+    qdq_q4k_kernel<<<grid_for(nsub, 1), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes), static_cast<uint4*>(a.scales));
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,
+                                cudaStream_t st) {
+  if (nx == 0 || ny == 0) return cudaSuccess;
+  selftest_div_kernel<<<kNumSMs * 8, 256, 0, st>>>(xs, nx, ys, ny, mismatches);
   return cudaGetLastError();
 }
 

@@ -44,6 +44,23 @@ def test_hardware_conversions_match_oracle_encoders():
     np.testing.assert_array_equal(e4m3.cpu().numpy(), want4)
 
 
+def test_reciprocal_based_division_is_the_ieee_quotient():
+    """The NVFP4 / Q4_K kernels divide through one exactly rounded reciprocal per block plus two fused
+    residual corrections; that must give the IEEE quotient bit for bit wherever it is used."""
+    rng = np.random.default_rng(11)
+    all_bf16 = (np.arange(0, 0x7F80, dtype=np.uint32) << 16).view(np.float32)          # every finite non-negative BF16
+    sb = np.array([oracle.e4m3_value(c) for c in range(1, 0x7F)], np.float32)
+    s_t = np.concatenate([np.float32(2.0) ** np.arange(-40, 20, 7), rng.uniform(1e-7, 1e-2, 24).astype(np.float32)])
+    ys = (s_t[:, None] * sb[None, :]).astype(np.float32).ravel()                       # NVFP4 divisors S = s_t * s_b
+    ys = ys[(ys >= 2.0 ** -60) & (ys <= 2.0 ** 60)]
+    xs = np.concatenate([all_bf16, rng.normal(0, 1, 20000).astype(np.float32)])        # plus FP32 numerators as in Q4_K
+    assert api.qf_selftest_div(torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()) == 0
+    ys2 = np.exp(rng.uniform(np.log(1e-9), np.log(1e3), 4000)).astype(np.float32)      # Q4_K style divisors
+    ys2 = np.concatenate([ys2, np.array([15.0, 63.0], np.float32)])
+    xs2 = np.concatenate([rng.normal(0, 1, 60000) * np.exp(rng.uniform(-12, 8, 60000)), np.arange(0, 16.5, 0.5)]).astype(np.float32)
+    assert api.qf_selftest_div(torch.from_numpy(xs2).cuda(), torch.from_numpy(ys2).cuda()) == 0
+
+
 @pytest.mark.parametrize("fmt,name", FMTS)
 @pytest.mark.parametrize("shape", [(1, 256), (3, 512), (37, 768), (129, 2304), (5, 8192)])
 def test_random_weights_small_and_ragged(fmt, name, shape):
