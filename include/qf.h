@@ -45,7 +45,8 @@ typedef enum {
   QF_ERR_CUDA = 6,      /* a CUDA runtime or driver call failed */
   QF_ERR_TIMEOUT = 7,   /* a bounded device-side wait expired (reported through the workspace status word) */
   QF_ERR_ARCH = 8,      /* the current device is not compute capability 10.x */
-  QF_ERR_DTYPE = 9      /* unknown output dtype */
+  QF_ERR_DTYPE = 9,     /* unknown output dtype */
+  QF_ERR_TOO_LARGE = 10 /* the problem needs more scratch than the built-in buffer of qf_fq_linear_fwd_noalloc */
 } qf_status_t;
 
 typedef enum { QF_DT_BF16 = 0, QF_DT_F32 = 1 } qf_dtype_t;
@@ -145,6 +146,34 @@ qf_status_t qf_fq_grouped_linear_bwd(const void* dY, const void* X, const void* 
                                      int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
                                      float* a_tscale, uint32_t flags, void* workspace,
                                      size_t workspace_bytes, void* stream);
+
+/* Allocation-free forward of the quantization-aware linear layer. (The paper has no counterpart:
+ * this is a packaging variant of qf_fq_linear_fwd for hosts that cannot hand the library a workspace.)
+ *
+ * Who needs it: code that runs where nobody may allocate device memory and where no spare buffer
+ * was planned for us — for example an extension loaded into a serving or training process whose
+ * memory planner reserved the whole device up front and forbids cudaMalloc (and the framework's own
+ * allocator) from extension code, or a hot loop that must never enter an allocator because a device
+ * allocation can synchronise the GPU. Such a caller still owns X, W and Y; what it lacks is a place
+ * for the two transient fake-quantized copies. Here that place is a buffer compiled into the
+ * library: QF_NOALLOC_SCRATCH_BYTES (32 MiB) of device memory per GPU, held by every GPU that loads
+ * libqf.so until the process exits.
+ *
+ * Same arithmetic, arguments and results as qf_fq_linear_fwd (no a_amax_out, no workspace). The call
+ * allocates nothing: no cudaMalloc / cudaFree / allocating library routine on any path.
+ *   Limit: 256 + round256(2*N*K) + round256(2*M*K) bytes must fit in QF_NOALLOC_SCRATCH_BYTES; larger
+ *          problems are rejected with QF_ERR_TOO_LARGE before anything is enqueued.
+ *   First call on each device: looks up the device address of the built-in buffer (once per device,
+ *          with that device current). Make that first call outside any stream capture.
+ *   Sharing: every call on a device uses the same buffer, which keeps the previous call's contents;
+ *          the call clears the words that must start at zero itself. Two calls whose GPU work can
+ *          overlap (different streams, no dependency between them) race on the buffer — serialise
+ *          them. A device-side timeout is not reported by this variant (there is no caller-visible
+ *          status word); use qf_fq_linear_fwd when that matters. */
+#define QF_NOALLOC_SCRATCH_BYTES (32u << 20)
+qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N,
+                                     int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
+                                     float* a_tscale, uint32_t flags, void* stream);
 
 /* Self-test hook for the hardware number-format conversions the kernels rely on: for each of n FP32
  * inputs (device), writes the E2M1 code (low nibble) into e2m1_out[i] and the E4M3 code of |x|

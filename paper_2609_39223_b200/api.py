@@ -25,8 +25,9 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc",
 ]
+NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
 class QfError(RuntimeError):
@@ -75,6 +76,9 @@ def lib() -> ctypes.CDLL:
                                                c_uint32, c_void_p, c_size_t, c_void_p]
         L.qf_selftest_cvt.restype = c_int
         L.qf_selftest_cvt.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
+        L.qf_fq_linear_fwd_noalloc.restype = c_int
+        L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
+                                               c_void_p, c_void_p, c_uint32, c_void_p]
         L.qf_selftest_div.restype = c_int
         L.qf_selftest_div.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p]
         _lib = L
@@ -254,3 +258,16 @@ def qf_selftest_div(xs: torch.Tensor, ys: torch.Tensor) -> int:
     out = torch.zeros(1, dtype=torch.int64, device=xs.device)
     _check(lib().qf_selftest_div(_ptr(xs), xs.numel(), _ptr(ys), ys.numel(), _ptr(out), _stream()), "qf_selftest_div")
     return int(out.item())
+
+
+def qf_fq_linear_fwd_noalloc(X, W, Y, wq_fmt: int, aq_fmt: int, *, w_tscale=None, a_tscale=None, flags: int = 0) -> torch.Tensor:
+    """Y = QDQ_a(X) . QDQ_w(W)^T through the entry point that allocates nothing: the caller passes the
+    output tensor, and the transient fake-quantized copies live in a 32 MiB buffer built into the
+    library (one per GPU, shared by all calls — do not let two such calls overlap on the GPU). Meant
+    for hosts that may not allocate device memory at call time; this wrapper therefore creates no tensor."""
+    X, W = _bf16(X, "X"), _bf16(W, "W")
+    M, K = X.shape
+    N = W.shape[0]
+    _check(lib().qf_fq_linear_fwd_noalloc(_ptr(X), _ptr(W), _ptr(Y), _dt(Y.dtype), M, N, K, wq_fmt, aq_fmt, _ptr(w_tscale),
+                                          _ptr(a_tscale), flags, _stream()), "qf_fq_linear_fwd_noalloc")
+    return Y

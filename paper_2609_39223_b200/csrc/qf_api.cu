@@ -221,6 +221,7 @@ const char* qf_status_string(qf_status_t s) {
     case QF_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case QF_ERR_ARCH: return "device is not compute capability 10.x";
     case QF_ERR_DTYPE: return "unknown output dtype";
+    case QF_ERR_TOO_LARGE: return "problem needs more scratch than the built-in buffer of the allocation-free entry point";
   }
   return "unknown status";
 }
@@ -353,6 +354,43 @@ qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8
   if (n < 0) return QF_ERR_SHAPE;
   if (qf_status_t s = check_arch()) return s;
   return cu(launch_selftest_cvt(in, n, e2m1_out, e4m3_out, static_cast<cudaStream_t>(stream)));
+}
+
+// ---- allocation-free variant -----------------------------------------------------------------------
+// Scratch for qf_fq_linear_fwd_noalloc lives in the library image itself. In host code the name of a
+// __device__ array is only a handle, not an address a kernel can use: the device address is
+// obtained per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[QF_NOALLOC_SCRATCH_BYTES];
+
+static qf_status_t noalloc_scratch_ptr(void** out) {
+  static void* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return QF_ERR_CUDA; }
+  if (dev < 0 || dev >= 64) return QF_ERR_CUDA;
+  void* p = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    // once per device, with that device current; racing first calls resolve to the same address
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return QF_ERR_CUDA; }
+    __atomic_store_n(&cached[dev], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return QF_OK;
+}
+
+qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N,
+                                     int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale,
+                                     uint32_t flags, void* stream) {
+  if (M < 0 || N < 0 || K < 0) return QF_ERR_SHAPE;
+  // size check in a form that cannot overflow: each operand copy must fit on its own first
+  const unsigned long long cap = QF_NOALLOC_SCRATCH_BYTES;
+  const unsigned long long n = static_cast<unsigned long long>(N), k = static_cast<unsigned long long>(K),
+                           m = static_cast<unsigned long long>(M);
+  if ((k != 0 && (n > cap / 2 / k || m > cap / 2 / k)) || linear_ws_bytes(M, N, K, 1) > cap) return QF_ERR_TOO_LARGE;
+  if (qf_status_t s = check_arch()) return s;
+  void* scratch = nullptr;
+  if (qf_status_t s = noalloc_scratch_ptr(&scratch)) return s;
+  return linear_fwd_impl(X, W, Y, y_dtype, nullptr, 1, M, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale, nullptr, flags, scratch,
+                         QF_NOALLOC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
 }
 
 qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream) {
