@@ -329,7 +329,7 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": KERNELS_PER_STEP * args.steps,
-            "roofline": {"bound": "tensor", "kernel": "gemm_kernel (tcgen05 BF16, 128x256x64 tiles)", "achieved": achieved,
+            "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel (tcgen05 cta_group::2 BF16, 256x256x64 tiles per CTA pair)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": None,
                          "peak_source": f"{peaks['source']} cuBLAS bf16 burst", "ms_per_launch": gemm_ms,
                          "frac_of_sustained": achieved / peaks["bf16_sustained"] if achieved else None,

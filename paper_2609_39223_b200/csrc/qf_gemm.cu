@@ -17,6 +17,7 @@
 // teardown (the producer first gives its outstanding copies a bounded chance to land), tensor
 // memory is released and the kernel returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "qf_common.cuh"
 
@@ -419,6 +420,247 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
+// =====================================================================================================
+// Two-CTA variant (cta_group::2): a cluster of two CTAs on neighbouring SMs computes a 256 x 256 output
+// tile with one M=256 MMA stream issued by the leader CTA. Each CTA stages only its own 128 rows of A
+// and its own 128 rows (half) of B, so the shared-memory operand traffic per SM is 64 B/clk instead of
+// the 96 B/clk of the one-CTA tile, and each holds its 128 accumulator rows in its own tensor memory.
+//   * both producers' TMA copies complete on the LEADER's full barrier (no multicast is used);
+//   * the leader frees a stage / publishes an accumulator with a tcgen05.commit multicast to the same
+//     barrier offset in both CTAs;
+//   * both CTAs' epilogue warps release the accumulator on the leader's barrier (remote arrive).
+// Plain (non-grouped) problems only.
+// =====================================================================================================
+
+constexpr int STAGES2 = 6;
+constexpr int A2_BYTES = BM * BK * 2;           // 16 KB: this CTA's 128 rows of A
+constexpr int B2_BYTES = (BN / 2) * BK * 2;     // 16 KB: this CTA's 128 rows of B
+constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+
+struct alignas(8) Barriers2 {
+  uint64_t full[STAGES2];       // leader's copy is the live one
+  uint64_t empty[STAGES2];      // one per CTA, released by the leader's commit multicast
+  uint64_t acc_full[2];         // one per CTA, published by the leader's commit multicast
+  uint64_t acc_empty[2];        // leader's copy is the live one: 8 arrivals (4 epilogue warps x 2 CTAs)
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA copy into this CTA's shared memory whose completion is counted on a barrier that may live in the
+// other CTA of the pair (cluster address). No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this offset in both CTAs of the pair once all MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ uint32_t instr_desc_pair() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+         (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+}
+
+__device__ __forceinline__ void decode_tile_pair(const KParams& p, int t, int& m0, int& n0) {
+  const int band = 8 * p.tiles_n;
+  const int bidx = t / band;
+  const int first_m = bidx * 8;
+  const int rows_in_band = min(8, p.tiles_m - first_m);
+  const int within = t - bidx * band;
+  m0 = (first_m + within % rows_in_band) * (2 * BM);
+  n0 = (within / rows_in_band) * BN;
+}
+
+template <bool A_MN, bool B_MN, typename OutT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  uint8_t* tiles_ptr = smem_raw + (tiles_base - raw);
+  Barriers2* bars = reinterpret_cast<Barriers2*>(tiles_ptr + STAGES2 * STAGE2_BYTES);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const bool leader = rank == 0;
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 8);
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(&bars->tmem_base), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                               // both CTAs' barriers exist before any remote access
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ===== TMA producer (both CTAs): own rows of A, own half of B, counted on the leader's barrier =====
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued = 0;
+      bool alive = true;
+      for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters) {
+        int m0, n0;
+        decode_tile_pair(p, t, m0, n0);
+        m0 += static_cast<int>(rank) * BM;
+        n0 += static_cast<int>(rank) * (BN / 2);
+        for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status)) { alive = false; break; }
+          const uint32_t full_local = smem_u32(&bars->full[stage]);
+          const uint32_t full_leader = mapa_shared(full_local, 0);
+          const uint32_t a_dst = tiles_base + stage * STAGE2_BYTES;
+          const uint32_t b_dst = a_dst + A2_BYTES;
+          if (leader) mbar_expect_tx(full_local, 2 * STAGE2_BYTES);      // both CTAs' bytes land on this barrier
+          if (A_MN) {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * 8192, &tmA, m0 + 64 * i, k, full_leader);
+          } else {
+            tma_load_2d_pair(a_dst, &tmA, k, m0, full_leader);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int i = 0; i < BN / 2 / 64; ++i) tma_load_2d_pair(b_dst + i * 8192, &tmB, n0 + 64 * i, k, full_leader);
+          } else {
+            tma_load_2d_pair(b_dst, &tmB, k, n0, full_leader);
+          }
+          ++issued;
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+      }
+      (void)issued;
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer (leader CTA only) =====
+    if (leader && lane == 0) {
+      const uint32_t idesc = instr_desc_pair<A_MN, B_MN>();
+      uint32_t stage = 0, phase = 0, local = 0;
+      bool alive = true;
+      for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters, ++local) {
+        const uint32_t buf = local & 1u;
+        const uint32_t use = local >> 1;
+        if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), (use & 1u) ^ 1u, abort_flag, p.status)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
+        uint32_t accumulate = 0;
+        for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
+          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
+          const uint64_t a_desc = smem_desc<A_MN>(a_addr);
+          const uint64_t b_desc = smem_desc<B_MN>(a_addr + A2_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            umma_bf16_pair(d_tmem, a_desc + kk * desc_k_step<A_MN>(), b_desc + kk * desc_k_step<B_MN>(), idesc, accumulate);
+            accumulate = 1;
+          }
+          umma_commit_pair(smem_u32(&bars->empty[stage]));
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        umma_commit_pair(smem_u32(&bars->acc_full[buf]));
+      }
+    }
+  } else {
+    // ===== epilogue (both CTAs): own 128 accumulator rows =====
+    const int quarter = warp & 3;
+    uint32_t local = 0;
+    bool alive = true;
+    for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters, ++local) {
+      int m0, n0;
+      decode_tile_pair(p, t, m0, n0);
+      m0 += static_cast<int>(rank) * BM;
+      const uint32_t buf = local & 1u;
+      const uint32_t use = local >> 1;
+      const bool got = mbar_wait(smem_u32(&bars->acc_full[buf]), use & 1u, abort_flag, p.status);
+      if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < static_cast<int>(p.Mo);
+      OutT* row_ptr = static_cast<OutT*>(p.C) + static_cast<int64_t>(row) * p.ldc;
+      const uint32_t taddr = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(quarter * 32) << 16);
+      const bool empty_k = p.Kc <= 0;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t acc[32];
+        tmem_ld32(taddr + c * 32, acc);
+        tmem_ld_wait();
+        if (c == BN / 32 - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->acc_empty[buf]), 0));
+        }
+        if (empty_k) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = 0u;
+        }
+        const int col0 = n0 + c * 32;
+        if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, p.accumulate != 0);
+      }
+    }
+  }
+
+  // ===== teardown: nobody leaves while the partner may still touch this CTA's memory or barriers =====
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -459,6 +701,24 @@ cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const KPara
   return cudaGetLastError();
 }
 
+template <bool A_MN, bool B_MN, typename OutT>
+cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid, cudaStream_t st) {
+  auto kern = gemm_pair_kernel<A_MN, B_MN, OutT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, kp);      // cluster shape (2,1,1) is a kernel attribute
+  return cudaGetLastError();
+}
+
+template <typename OutT>
+cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid,
+                               cudaStream_t st) {
+  if (!a.a_mn_major && !a.b_mn_major) return launch_pair_t<false, false, OutT>(tmA, tmB, kp, grid, st);
+  if (!a.a_mn_major && a.b_mn_major) return launch_pair_t<false, true, OutT>(tmA, tmB, kp, grid, st);
+  if (a.a_mn_major && a.b_mn_major) return launch_pair_t<true, true, OutT>(tmA, tmB, kp, grid, st);
+  return launch_pair_t<true, false, OutT>(tmA, tmB, kp, grid, st);
+}
+
 template <typename OutT>
 cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid,
                           cudaStream_t st) {
@@ -470,8 +730,47 @@ cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUten
 
 }  // namespace
 
+// Two-CTA path: plain problems whose output has at least one full 256-row pair tile.
+cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
+  KParams kp{};
+  kp.C = a.C;
+  kp.Mo = a.Mo;
+  kp.No = a.No;
+  kp.Kc = a.Kc;
+  kp.ldc = a.ldc;
+  kp.c_dtype = a.c_dtype;
+  kp.accumulate = a.accumulate ? 1 : 0;
+  kp.status = a.status_word;
+  kp.tiles_m = static_cast<int>((a.Mo + 2 * BM - 1) / (2 * BM));
+  kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
+  kp.num_tiles = kp.tiles_m * kp.tiles_n;
+  CUtensorMap tmA, tmB;
+  bool ok;
+  if (a.a_mn_major) ok = make_map(&tmA, a.A, a.Kc, a.Mo, a.lda, 64, BK);
+  else ok = make_map(&tmA, a.A, a.Mo, a.Kc, a.lda, BK, BM);
+  if (!ok) return cudaErrorInvalidValue;
+  if (a.b_mn_major) ok = make_map(&tmB, a.B, a.Kc, a.No, a.ldb, 64, BK);
+  else ok = make_map(&tmB, a.B, a.No, a.Kc, a.ldb, BK, BN / 2);
+  if (!ok) return cudaErrorInvalidValue;
+  const int clusters = kp.num_tiles < kNumSMs / 2 ? kp.num_tiles : kNumSMs / 2;
+  const int grid = 2 * clusters;
+  if (a.c_dtype == QF_DT_F32) return launch_pair_majors<float>(a, tmA, tmB, kp, grid, st);
+  return launch_pair_majors<__nv_bfloat16>(a, tmA, tmB, kp, grid, st);
+}
+
+static int pair_mode() {
+  // QF_GEMM_PAIR=0 forces the one-CTA kernel (A/B comparison in profiling runs); default: two-CTA when it applies
+  static int mode = -1;
+  if (mode < 0) {
+    const char* e = getenv("QF_GEMM_PAIR");
+    mode = (e && e[0] == '0') ? 0 : 1;
+  }
+  return mode;
+}
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
+  if (a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode()) return launch_gemm_pair(a, st);
   KParams kp{};
   kp.C = a.C;
   kp.Mo = a.Mo;
