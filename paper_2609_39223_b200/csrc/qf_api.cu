@@ -72,9 +72,8 @@ qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t col
     if (tscale_given) {
       q.tscale_in = tscale_user;
     } else {
-      if (cudaError_t e = launch_amax(src, rows * cols, header + amax_word, st)) return cu(e);
-      q.amax_bits = header + amax_word;
       q.tscale_out = tscale_user ? tscale_user : reinterpret_cast<float*>(header + scale_word);
+      return cu(launch_qdq_nvfp4_derive(q, header, amax_word, st));
     }
   }
   return cu(launch_qdq(q, st));
@@ -277,9 +276,8 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
     if (need_amax) {
       uint32_t* header = static_cast<uint32_t*>(workspace);
       if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
-      if (cudaError_t e = launch_amax(in, rows * cols, header + kWsAmaxW, st)) return cu(e);
-      q.amax_bits = header + kWsAmaxW;
       q.tscale_out = tensor_scale;
+      return cu(launch_qdq_nvfp4_derive(q, header, kWsAmaxW, st));
     } else {
       q.tscale_in = tensor_scale;
     }

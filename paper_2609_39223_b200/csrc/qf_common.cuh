@@ -89,11 +89,13 @@ struct QdqArgs {
   const float* tscale_in;        // NVFP4: tensor scale to read (device), or
   const uint32_t* amax_bits;     // NVFP4: tensor amax as FP32 bits (device) to derive it from
   float* tscale_out;             // NVFP4: where the derived scale is written (nullable)
+  bool reverse;                  // walk the tensor back to front (after an amax pass: L2 holds the tail)
 };
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);
 cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStream_t st);
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st);
+cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st);
 cudaError_t launch_dequant(int fmt, const void* codes, const void* scales, const float* tscale, int64_t rows,
                            int64_t cols, void* out, cudaStream_t st);
 cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,
