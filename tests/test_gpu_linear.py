@@ -172,3 +172,57 @@ def test_grouped_empty_expert_gives_zero_dw():
     assert torch.count_nonzero(dw[1]) == 0
     _close(dw, dw_ref, "grouped dW")
     _close(dx, dx_ref, "grouped dX")
+
+
+def test_full_size_nvfp4_weight_only_32k_tokens_sampled_rows():
+    """One 32K-token sequence through an up projection, NVFP4 weights, unquantized activations:
+    X 32768x4096, W 14336x4096 (and the matching down-projection shape for the backward operands)."""
+    M, N, K = 32768, 14336, 4096
+    c = synth.linear_case(M, N, K, seed=4, device="cuda", outlier_channels=0)
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    wts = torch.zeros(1, device="cuda")
+    y = api.qf_fq_linear_fwd(c.X, c.W, api.FMT_NVFP4, api.FMT_NONE, y_dtype=torch.bfloat16, ws=ws, w_tscale=wts)
+    dx, dw = api.qf_fq_linear_bwd(c.dY, c.X, c.W, api.FMT_NVFP4, api.FMT_NONE, dx_dtype=torch.bfloat16, dw_dtype=torch.float32, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    rng = np.random.default_rng(4)
+    rows = np.sort(rng.choice(M, 16, replace=False)); rows[0] = 0; rows[-1] = M - 1
+    wb = torch_to_bits(c.W)
+    qw = oracle.qdq(api.FMT_NVFP4, wb)
+    assert wts.item() == np.float32(qw["tensor_scale"])
+    w_hat = qw["out"]
+    xb = torch_to_bits(c.X[torch.from_numpy(rows).cuda()])
+    y_ref = oracle.matmul_fwd(xb, w_hat)
+    # BF16 outputs: compare with the tolerance plus one BF16 rounding of the reference
+    got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert np.all(np.abs(got - y_ref) <= TOL * _rms(y_ref) + np.abs(y_ref) * 2.0 ** -8)
+    dyb = torch_to_bits(c.dY[torch.from_numpy(rows).cuda()])
+    dx_ref = oracle.matmul_dgrad(dyb, w_hat)
+    gdx = dx[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert np.all(np.abs(gdx - dx_ref) <= TOL * _rms(dx_ref) + np.abs(dx_ref) * 2.0 ** -8)
+    n_idx = np.sort(rng.choice(N, 8, replace=False)); n_idx[0] = 0; n_idx[-1] = N - 1
+    dw_ref = oracle.matmul_wgrad(torch_to_bits(c.dY), torch_to_bits(c.X), n_idx)
+    _close(dw[torch.from_numpy(n_idx).cuda()], dw_ref, "dW rows")
+
+
+def test_full_size_moe_grouped_mxfp4_sampled_experts():
+    """128 experts, hidden 2048, expert MLP 768, 16384 tokens routed top-8: the gate/up projection
+    (N=768, K=2048) forward and backward over all 131072 routed rows; three experts checked in full."""
+    tokens, E, top_k, H, F = 16384, 128, 8, 2048, 768
+    r = synth.moe_routing(tokens, E, top_k, seed=0)
+    assert abs(int(r.counts.sum()) - tokens * top_k) == 0 and int(r.counts.min()) > 0
+    X = synth.randn_bf16((tokens, H), 1.0, 1)
+    Xp = synth.gather_rows(X, r.token_of_row).cuda()
+    W = synth.randn_bf16((E, F, H), 0.02, 2, device="cuda")
+    dYp = synth.randn_bf16((Xp.shape[0], F), 1e-3, 3, device="cuda")
+    dYp[(r.token_of_row < 0).cuda()] = 0
+    offs = r.group_offsets.cuda()
+    fmt = api.FMT_MXFP4
+    y = api.qf_fq_grouped_linear_fwd(Xp, W, offs, fmt, fmt, y_dtype=torch.float32)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp, Xp, W, offs, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    for g in (0, 57, 127):
+        a, b = int(r.group_offsets[g]), int(r.group_offsets[g + 1])
+        xb, wb, dyb = torch_to_bits(Xp[a:b]), torch_to_bits(W[g]), torch_to_bits(dYp[a:b])
+        _close(y[a:b], oracle.fq_linear_fwd(xb, wb, fmt, fmt), f"expert {g} Y")
+        dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, fmt, fmt)
+        _close(dx[a:b], dx_ref, f"expert {g} dX")
+        _close(dw[g], dw_ref, f"expert {g} dW")
