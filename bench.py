@@ -164,6 +164,90 @@ def run_reference(args):
 
 
 # -------------------------------------------------------------------------------------------------
+# the other named workloads (parity-test cases; measured on request with --sections ...,configs)
+# -------------------------------------------------------------------------------------------------
+
+def _time_ms(torch, fn, reps=5, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def measure_other_workloads(torch, api, synth, dev, peaks):
+    out = {}
+    # 1: NVFP4 QDQ of 2048x2048 weights, a rotating set of 32 matrices (268 MB, more than twice L2)
+    mats = [synth.weight_with_outliers(2048, 2048, seed=i, device=dev) for i in range(32)]
+    o = torch.empty_like(mats[0]); c = torch.empty((2048, 1024), dtype=torch.uint8, device=dev)
+    sc = torch.empty((2048, 128), dtype=torch.uint8, device=dev); wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
+    ms = _time_ms(torch, lambda: [api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq) for m in mats]) / 32
+    out["nvfp4_qdq_2048x2048"] = {"us_per_matrix": ms * 1e3, "gbs": 19136516 / (ms * 1e-3) / 1e9,
+                                  "note": "32 distinct matrices in rotation (cold L2); includes the amax pre-pass and launch overheads"}
+    del mats
+    # 3: Q4_K QDQ over all linear weights of the 32-layer dense decoder (one layer's buffers reused 32 times)
+    layer = [synth.randn_bf16((r, cc), 0.02, 100 + i, device=dev) for i, (_, r, cc) in enumerate(synth.DENSE_DECODER_LAYER)]
+    outs = [torch.empty_like(w) for w in layer]
+    codes = [torch.empty((w.shape[0], w.shape[1] // 2), dtype=torch.uint8, device=dev) for w in layer]
+    scs = [torch.empty(api.scales_shape(api.FMT_Q4_K, *w.shape), dtype=torch.uint8, device=dev) for w in layer]
+
+    def q4k_all():
+        for _ in range(synth.DENSE_DECODER_LAYERS):
+            for w, oo, cc, ss in zip(layer, outs, codes, scs):
+                api.qf_qdq(api.FMT_Q4_K, w, out=oo, codes=cc, scales=ss, ws=wsq)
+    ms = _time_ms(torch, q4k_all, reps=2, warm=1)
+    elems = synth.dense_decoder_layer_elems() * synth.DENSE_DECODER_LAYERS
+    out["q4k_qdq_dense_decoder_32_layers"] = {"ms": ms, "elements": elems, "gbs": elems * 4.5625 / (ms * 1e-3) / 1e9,
+                                              "frac_of_measured_hbm": elems * 4.5625 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    del layer, outs, codes, scs
+    # 4: NVFP4 weight-only linear, one 32K-token sequence, up and down projections, fwd + bwd
+    Mt = 32768
+    tot_ms, tot_fl = 0.0, 0.0
+    for (Nn, Kk) in ((14336, 4096), (4096, 14336)):
+        cse = synth.linear_case(Mt, Nn, Kk, seed=4, device=dev, outlier_channels=0)
+        ws4 = api.workspace(api.OP_LINEAR_BWD, Mt, Nn, Kk, device=dev)
+        Y = torch.empty((Mt, Nn), dtype=torch.bfloat16, device=dev); dX = torch.empty((Mt, Kk), dtype=torch.bfloat16, device=dev)
+        dW = torch.empty((Nn, Kk), dtype=torch.float32, device=dev); wts = torch.zeros(1, device=dev)
+
+        def f4():
+            api.qf_fq_linear_fwd(cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, Y=Y, w_tscale=wts)
+            api.qf_fq_linear_bwd(cse.dY, cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, dX=dX, dW=dW, w_tscale=wts)
+        tot_ms += _time_ms(torch, f4, reps=3, warm=2)
+        tot_fl += 3 * 2.0 * Mt * Nn * Kk
+        del cse, ws4, Y, dX, dW
+    out["nvfp4_weight_only_linear_32k_tokens_up_down"] = {"ms": tot_ms, "tflops": tot_fl / (tot_ms * 1e-3) / 1e12,
+                                                           "frac_of_2250_datasheet": tot_fl / (tot_ms * 1e-3) / 1e12 / 2250.0}
+    # 5: MoE grouped MXFP4 W4A4: 128 experts, top-8 of 16384 tokens, gate + up + down, fwd + bwd
+    tokens, E, top_k, H, F = 16384, 128, 8, 2048, 768
+    r = synth.moe_routing(tokens, E, top_k, seed=0)
+    rows = int(r.group_offsets[-1]); offs = r.group_offsets.to(dev)
+    fmt = api.FMT_MXFP4
+    tot_ms = 0.0
+    for (Nn, Kk, times) in ((F, H, 2), (H, F, 1)):
+        Xp = synth.randn_bf16((rows, Kk), 1.0, 5, device=dev); Xp[(r.token_of_row < 0).to(dev)] = 0
+        Wg = synth.randn_bf16((E, Nn, Kk), 0.02, 6, device=dev)
+        dYp = synth.randn_bf16((rows, Nn), 1e-3, 7, device=dev); dYp[(r.token_of_row < 0).to(dev)] = 0
+        ws5 = api.workspace(api.OP_GROUPED_BWD, rows, Nn, Kk, E, device=dev)
+        Y = torch.empty((rows, Nn), dtype=torch.bfloat16, device=dev); dX = torch.empty((rows, Kk), dtype=torch.bfloat16, device=dev)
+        dW = torch.empty((E, Nn, Kk), dtype=torch.float32, device=dev)
+
+        def f5():
+            api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
+            api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dW)
+        tot_ms += times * _time_ms(torch, f5, reps=3, warm=2)
+        del Xp, Wg, dYp, ws5, Y, dX, dW
+    fl = 3 * 3 * 2.0 * tokens * top_k * H * F
+    out["moe_grouped_mxfp4_128_experts"] = {"ms": tot_ms, "tflops": fl / (tot_ms * 1e-3) / 1e12, "routed_rows": tokens * top_k,
+                                            "padded_rows": rows, "frac_of_2250_datasheet": fl / (tot_ms * 1e-3) / 1e12 / 2250.0}
+    return out
+
+
+# -------------------------------------------------------------------------------------------------
 # our arm
 # -------------------------------------------------------------------------------------------------
 
@@ -343,6 +427,12 @@ def run_ours(args):
                "sample": f"fwd+dX+dW on a [{m_rows},{K}] x [{n_rows},{K}] slice of the workload, QDQ of both slices "
                          f"included, {dt:.1f} s"}
 
+    other = None
+    if rank == 0 and world == 1 and "configs" in sections:
+        del X, W, dY, Y, dX, dW, ws
+        torch.cuda.empty_cache()
+        other = measure_other_workloads(torch, api, synth, dev, peaks)
+
     if rank == 0:
         clocks = clk.summary()
         peak = peaks["bf16_burst"]
@@ -365,6 +455,8 @@ def run_ours(args):
             "cpu_baseline": cpu,
             "qdq_gbs": qdq,
         }
+        if other is not None:
+            line["other_workloads"] = other
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -377,7 +469,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sections", default=",".join(SECTIONS),
-                    help="extra measurements beside the headline: roofline,qdq,e2e,cpu (empty string: none)")
+                    help="extra measurements beside the headline: roofline,qdq,e2e,cpu (default), configs = the other "
+                         "named workloads (empty string: none)")
     ap.add_argument("--shape", default=None, help="M,N,K of a smaller case (profiler captures only)")
     args = ap.parse_args()
     if args.shape:

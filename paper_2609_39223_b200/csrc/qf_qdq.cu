@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restri
       const int64_t lin = first + base + u * stride;
       // reverse: walk whole warps' worth of units from the end (block pairs of lanes stay adjacent)
       const int64_t i = reverse ? (nunits_up - 32 - (lin - lane)) + lane : lin;
-      ok[u] = i < nunits;
+      ok[u] = lin < nunits_up && i < nunits;      // lin past the end would map to a negative index in reverse
       v[u][0] = ok[u] ? ld_chunk(in + 2 * i) : make_uint4(0, 0, 0, 0);
       v[u][1] = ok[u] ? ld_chunk(in + 2 * i + 1) : make_uint4(0, 0, 0, 0);
     }

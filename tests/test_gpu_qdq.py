@@ -165,3 +165,39 @@ def test_full_size_q4k_decoder_matrices(name):
 def test_full_size_mxfp4_activation():
     x = synth.activations_with_outlier_channels(8192, 4096, seed=0)
     _compare(api.FMT_MXFP4, torch_to_bits(x))
+
+
+def _guarded(nbytes, dtype, shape):
+    """A tensor carved out of the middle of a larger byte buffer whose margins are filled with a canary."""
+    pad = 1 << 16
+    raw = torch.full((nbytes + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+    view = raw[pad:pad + nbytes].view(dtype).view(shape)
+    return raw, view, pad
+
+
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_large_ragged_tensor_stays_inside_its_buffers(fmt, name):
+    """A tensor large enough that the capped grid loops several times with a ragged last iteration:
+    outputs must be bit-exact and nothing may be written outside the output buffers."""
+    rows, cols = 9001, 4352
+    w = synth.randn_bf16((rows, cols), 0.02, 17, device="cuda")
+    n = rows * cols
+    raw_o, out, pad = _guarded(n * 2, torch.bfloat16, (rows, cols))
+    raw_c, codes, _ = _guarded(n // 2, torch.uint8, (rows, cols // 2))
+    sshape = api.scales_shape(fmt, rows, cols)
+    raw_s, scales, _ = _guarded(int(np.prod(sshape)), torch.uint8, sshape)
+    g = api.qf_qdq(fmt, w, out=out, codes=codes, scales=scales)          # NVFP4: derived scale (amax pass + reverse walk)
+    torch.cuda.synchronize()
+    for raw in (raw_o, raw_c, raw_s):
+        assert bool((raw[:pad] == 0xA5).all()) and bool((raw[-pad:] == 0xA5).all())
+    o = oracle.qdq(fmt, torch_to_bits(w))
+    np.testing.assert_array_equal(torch_to_bits(out), o["out"])
+    np.testing.assert_array_equal(codes.cpu().numpy(), o["codes"])
+    np.testing.assert_array_equal(scales.cpu().numpy(), o["scales"])
+    if fmt == api.FMT_NVFP4:
+        out.zero_()
+        api.qf_qdq(fmt, w, out=out, codes=codes, scales=scales, tensor_scale=g["tensor_scale"])   # forward walk
+        torch.cuda.synchronize()
+        for raw in (raw_o, raw_c, raw_s):
+            assert bool((raw[:pad] == 0xA5).all()) and bool((raw[-pad:] == 0xA5).all())
+        np.testing.assert_array_equal(torch_to_bits(out), o["out"])
