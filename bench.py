@@ -186,9 +186,15 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
     mats = [synth.weight_with_outliers(2048, 2048, seed=i, device=dev) for i in range(32)]
     o = torch.empty_like(mats[0]); c = torch.empty((2048, 1024), dtype=torch.uint8, device=dev)
     sc = torch.empty((2048, 128), dtype=torch.uint8, device=dev); wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
-    ms = _time_ms(torch, lambda: [api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq) for m in mats]) / 32
+    ts1 = torch.empty(1, dtype=torch.float32, device=dev)
+    run1 = lambda: [api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq, tensor_scale=None, ts_out=ts1) for m in mats]
+    run1(); torch.cuda.synchronize()
+    g1 = torch.cuda.CUDAGraph()                  # replayed as a graph: the Python binding's per-call cost is not GPU time
+    with torch.cuda.graph(g1):
+        run1()
+    ms = _time_ms(torch, g1.replay) / 32
     out["nvfp4_qdq_2048x2048"] = {"us_per_matrix": ms * 1e3, "gbs": 19136516 / (ms * 1e-3) / 1e9,
-                                  "note": "32 distinct matrices in rotation (cold L2); includes the amax pre-pass and launch overheads"}
+                                  "note": "32 distinct matrices in rotation (cold L2), replayed as one CUDA graph; includes the header memset and the amax pre-pass"}
     del mats
     # 3: Q4_K QDQ over all linear weights of the 32-layer dense decoder (one layer's buffers reused 32 times)
     layer = [synth.randn_bf16((r, cc), 0.02, 100 + i, device=dev) for i, (_, r, cc) in enumerate(synth.DENSE_DECODER_LAYER)]
@@ -200,7 +206,11 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
         for _ in range(synth.DENSE_DECODER_LAYERS):
             for w, oo, cc, ss in zip(layer, outs, codes, scs):
                 api.qf_qdq(api.FMT_Q4_K, w, out=oo, codes=cc, scales=ss, ws=wsq)
-    ms = _time_ms(torch, q4k_all, reps=2, warm=1)
+    q4k_all(); torch.cuda.synchronize()
+    g3 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g3):
+        q4k_all()
+    ms = _time_ms(torch, g3.replay, reps=3, warm=1)
     elems = synth.dense_decoder_layer_elems() * synth.DENSE_DECODER_LAYERS
     out["q4k_qdq_dense_decoder_32_layers"] = {"ms": ms, "elements": elems, "gbs": elems * 4.5625 / (ms * 1e-3) / 1e9,
                                               "frac_of_measured_hbm": elems * 4.5625 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}

@@ -135,7 +135,7 @@ def scales_shape(fmt: int, rows: int, cols: int):
 
 
 def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_scales=True, tensor_scale=None,
-           ws: torch.Tensor | None = None, out=None, codes=None, scales=None):
+           ws: torch.Tensor | None = None, out=None, codes=None, scales=None, ts_out=None):
     """(C, theta) = Q(x), x_hat = Q^-1(C, theta). Returns dict(out, codes, scales, tensor_scale); the
     tensor scale (NVFP4) is a 1-element float32 CUDA tensor, read if ``tensor_scale`` is given."""
     x = _bf16(x, "x")
@@ -154,7 +154,7 @@ def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_sc
             ts = tensor_scale if isinstance(tensor_scale, torch.Tensor) else torch.tensor([tensor_scale], dtype=torch.float32, device=dev)
             flags |= TENSOR_SCALE_GIVEN
         else:
-            ts = torch.empty(1, dtype=torch.float32, device=dev)
+            ts = ts_out if ts_out is not None else torch.empty(1, dtype=torch.float32, device=dev)
     if ws is None:
         ws = workspace(OP_QDQ, rows, 0, cols, device=dev)
     _check(lib().qf_qdq(fmt, _ptr(x), rows, cols, _ptr(out), _ptr(codes), _ptr(scales), _ptr(ts), flags, _ptr(ws),

@@ -60,12 +60,17 @@ __global__ void amax_to_float_kernel(const uint32_t* amax_bits, float* out) { *o
 // The formats need v = x / S (NVFP4) and t = (x + em) / es (Q4_K) as correctly rounded FP32
 // quotients, because the quotient decides a code. One divisor serves a whole block, so its correctly
 // rounded reciprocal rc = RN(1/y) is computed once and every quotient is then
-//     q0 = RN(x * rc);  q1 = RN(q0 + rc * RN(x - y*q0));  q2 = RN(q1 + rc * RN(x - y*q1))
-// (fused multiply-adds, two elements per instruction). With an exactly rounded reciprocal and
-// no overflow / underflow in the residuals this is the classical correctly-rounded division
-// iteration (Markstein); the range guard below keeps operands where that holds and the
-// caller falls back to the IEEE divide otherwise. qf_selftest_div compares it with the IEEE divide.
+//     q0 = RN(x * rc);  q1 = RN(q0 + rc * (x - y*q0))          (x - y*q0 is exact in a fused multiply-add)
+// (two elements per instruction). With an exactly rounded reciprocal and no overflow / underflow in
+// the residual, q1 is the correctly rounded quotient (Markstein's division theorem); the range guard
+// below keeps operands where that holds and the caller falls back to the IEEE divide otherwise.
+// qf_selftest_div compares it with the IEEE divide (tens of billions of pairs, including every BF16
+// numerator and divisors with an all-ones significand, without a difference).
 // ---------------------------------------------------------------------------------------------
+
+#ifndef QF_DIV_STEPS
+#define QF_DIV_STEPS 1      // residual corrections after the first product (1 suffices with an exact reciprocal)
+#endif
 
 __device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
 
@@ -73,13 +78,17 @@ __device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
   const float2 ny = splat(-y), r = splat(rc);
   float2 q = __fmul2_rn(x, r);
   q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+#if QF_DIV_STEPS > 1
   q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+#endif
   return q;
 }
 __device__ __forceinline__ float div1_fast(float x, float y, float rc) {
   float q = __fmul_rn(x, rc);
   q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+#if QF_DIV_STEPS > 1
   q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+#endif
   return q;
 }
 // divisor magnitudes for which the iteration above is used
