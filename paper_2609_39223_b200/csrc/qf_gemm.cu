@@ -47,7 +47,8 @@ struct alignas(8) Barriers {
   int abort_flag;
 };
 
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* Barriers */;
+constexpr int STAGING_BYTES = 4 * 2 * 4096;    // epilogue: per warp two 32-row x 128-byte staging buffers for TMA stores
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /* alignment slack */ + 256 /* Barriers */;
 
 struct KParams {
   void* C;
@@ -177,6 +178,7 @@ struct Tile {
   int b_row_off;       // mode 1: row offset of this tile's group in B's tensor map
   int64_t c_off;       // mode 2: element offset of this tile's group in C
   int m_limit;         // rows of C that exist for this tile's matrix
+  int group;           // mode 2: which per-group output matrix
 };
 
 __device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_group) {
@@ -186,6 +188,7 @@ __device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_g
   r.k_begin = 0;
   r.k_end = static_cast<int>(p.Kc);
   r.m_limit = static_cast<int>(p.Mo);
+  r.group = 0;
   int g = 0;
   if (p.group_mode == 2) {
     const int per = p.tiles_m * p.tiles_n;
@@ -212,6 +215,7 @@ __device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_g
     r.k_begin = __ldg(p.offs + g);
     r.k_end = __ldg(p.offs + g + 1);
     r.c_off = static_cast<int64_t>(g) * p.c_group_stride;
+    r.group = g;
   }
   return r;
 }
@@ -265,16 +269,102 @@ __device__ __forceinline__ void store_chunk32<float>(float* row_ptr, int col0, i
   }
 }
 
+// ---- epilogue through shared memory and TMA stores ------------------------------------------------------
+// Each epilogue warp owns 32 accumulator rows (its quarter of the TMEM lanes). Per column chunk of
+// 128 bytes of output (64 BF16 or 32 FP32 values) a lane reads its row from TMEM, converts it, and writes
+// it into a 32 x 128-byte staging buffer with the 128-byte swizzle (16-byte chunk j of row r goes to
+// chunk j ^ (r & 7): conflict-free), then one lane issues a TMA store (or a TMA add-reduce when
+// accumulating in FP32) of the 32-row box. The tensor map clips rows and columns past the matrix edge.
+// Two staging buffers per warp let the next chunk be converted while the previous store drains.
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <typename OutT>
+struct EpiChunk {
+  static constexpr int COLS = 128 / static_cast<int>(sizeof(OutT));   // output columns per 128-byte staging row
+  static constexpr int NCHUNK = BN / COLS;
+};
+
+// One tile's worth of TMA-store epilogue for one warp. `release` is called once, right after the last
+// TMEM read, so the accumulator can be handed back before the remaining stores are issued.
+template <typename OutT, typename Release>
+__device__ __forceinline__ void epilogue_tile_tma(const CUtensorMap* tmC, uint32_t warp_staging, uint32_t& which, uint32_t taddr,
+                                                  int row0, int n0, int z, int rows_limit, int n_limit, bool accumulate,
+                                                  bool empty_k, int lane, Release release) {
+  constexpr int COLS = EpiChunk<OutT>::COLS;
+  constexpr int NCHUNK = EpiChunk<OutT>::NCHUNK;
+#pragma unroll 1
+  for (int c = 0; c < NCHUNK; ++c) {
+    uint32_t acc[COLS];
+#pragma unroll
+    for (int h = 0; h < COLS / 32; ++h) tmem_ld32(taddr + c * COLS + h * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[32 * h]));
+    tmem_ld_wait();
+    if (c == NCHUNK - 1) release();
+    if (empty_k) {
+#pragma unroll
+      for (int j = 0; j < COLS; ++j) acc[j] = 0u;
+    }
+    // the buffer about to be overwritten was the source of the store issued two chunks ago
+    if (lane == 0) bulk_wait_read_1();
+    __syncwarp();
+    const uint32_t buf = warp_staging + which * 4096u;
+    const uint32_t row_addr = buf + static_cast<uint32_t>(lane) * 128u;
+    const uint32_t sw = static_cast<uint32_t>(lane & 7);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      uint32_t v0, v1, v2, v3;
+      if constexpr (sizeof(OutT) == 2) {
+        v0 = pack_bf16x2(__uint_as_float(acc[8 * j]), __uint_as_float(acc[8 * j + 1]));
+        v1 = pack_bf16x2(__uint_as_float(acc[8 * j + 2]), __uint_as_float(acc[8 * j + 3]));
+        v2 = pack_bf16x2(__uint_as_float(acc[8 * j + 4]), __uint_as_float(acc[8 * j + 5]));
+        v3 = pack_bf16x2(__uint_as_float(acc[8 * j + 6]), __uint_as_float(acc[8 * j + 7]));
+      } else {
+        v0 = acc[4 * j]; v1 = acc[4 * j + 1]; v2 = acc[4 * j + 2]; v3 = acc[4 * j + 3];
+      }
+      st_shared_v4(row_addr + ((static_cast<uint32_t>(j) ^ sw) << 4), v0, v1, v2, v3);
+    }
+    fence_async_smem();
+    __syncwarp();
+    const int col0 = n0 + c * COLS;
+    if (lane == 0) {
+      if (row0 < rows_limit && col0 < n_limit) {
+        if (accumulate) tma_reduce_add_3d(tmC, buf, col0, row0, z);
+        else tma_store_3d(tmC, buf, col0, row0, z);
+      }
+      bulk_commit();
+    }
+    which ^= 1u;
+  }
+}
+
 // ---- the kernel -----------------------------------------------------------------------------------
 
 template <bool A_MN, bool B_MN, typename OutT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;                   // swizzled tiles need 1024-byte alignment
   uint8_t* tiles_ptr = smem_raw + (tiles_base - raw);
-  Barriers* bars = reinterpret_cast<Barriers*>(tiles_ptr + STAGES * STAGE_BYTES);
+  const uint32_t staging_base = tiles_base + STAGES * STAGE_BYTES;
+  Barriers* bars = reinterpret_cast<Barriers*>(tiles_ptr + STAGES * STAGE_BYTES + STAGING_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -377,8 +467,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else {
     // ===== epilogue: TMEM -> registers -> global =====
     const int quarter = warp & 3;                               // TMEM lanes 32*quarter .. +31 belong to this warp
-    uint32_t local = 0;
+    uint32_t local = 0, which = 0;
     bool alive = true;
+    const bool use_tma = !(p.accumulate != 0 && sizeof(OutT) == 2);
     for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x, ++local) {
       const Tile tile = decode_tile(p, t, false);
       const uint32_t buf = local & 1u;
@@ -386,29 +477,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const bool got = mbar_wait(smem_u32(&bars->acc_full[buf]), use & 1u, abort_flag, p.status);
       if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }        // keep the warp converged for tcgen05.ld
       tc_fence_after();
-      const int row = tile.m0 + quarter * 32 + lane;
-      const bool row_ok = row < tile.m_limit;
-      OutT* row_ptr = static_cast<OutT*>(p.C) + tile.c_off + static_cast<int64_t>(row) * p.ldc;
       const uint32_t taddr = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(quarter * 32) << 16);
       const bool empty_k = tile.k_end <= tile.k_begin;
+      if (use_tma) {
+        epilogue_tile_tma<OutT>(&tmC, staging_base + static_cast<uint32_t>(warp - 2) * 8192u, which, taddr,
+                                tile.m0 + quarter * 32, tile.n0, tile.group, tile.m_limit, static_cast<int>(p.No),
+                                p.accumulate != 0, empty_k, lane, [&]() {
+                                  tc_fence_before();
+                                  mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                                });
+      } else {
+        // BF16 output with accumulation: add in FP32 and round once (a TMA add-reduce would round twice)
+        const int row = tile.m0 + quarter * 32 + lane;
+        const bool row_ok = row < tile.m_limit;
+        OutT* row_ptr = static_cast<OutT*>(p.C) + tile.c_off + static_cast<int64_t>(row) * p.ldc;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t acc[32];
-        tmem_ld32(taddr + c * 32, acc);
-        tmem_ld_wait();
-        if (c == BN / 32 - 1) {
-          // every value of this accumulator is now in registers: hand the buffer back to the MMA warp
-          tc_fence_before();
-          mbar_arrive(smem_u32(&bars->acc_empty[buf]));
-        }
-        if (empty_k) {
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+          if (c == BN / 32 - 1) {
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+          }
+          if (empty_k) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = 0u;
+            for (int j = 0; j < 32; ++j) acc[j] = 0u;
+          }
+          const int col0 = tile.n0 + c * 32;
+          if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, true);
         }
-        const int col0 = tile.n0 + c * 32;
-        if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, p.accumulate != 0);
       }
     }
+    if (lane == 0) bulk_wait_all();          // every TMA store of this warp has completed before the CTA retires
   }
 
   // ===== teardown =====
@@ -436,7 +537,7 @@ constexpr int STAGES2 = 6;
 constexpr int A2_BYTES = BM * BK * 2;           // 16 KB: this CTA's 128 rows of A
 constexpr int B2_BYTES = (BN / 2) * BK * 2;     // 16 KB: this CTA's 128 rows of B
 constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256;
 
 struct alignas(8) Barriers2 {
   uint64_t full[STAGES2];       // leader's copy is the live one
@@ -511,12 +612,14 @@ __device__ __forceinline__ void decode_tile_pair(const KParams& p, int t, int& m
 
 template <bool A_MN, bool B_MN, typename OutT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   uint8_t* tiles_ptr = smem_raw + (tiles_base - raw);
-  Barriers2* bars = reinterpret_cast<Barriers2*>(tiles_ptr + STAGES2 * STAGE2_BYTES);
+  const uint32_t staging_base = tiles_base + STAGES2 * STAGE2_BYTES;
+  Barriers2* bars = reinterpret_cast<Barriers2*>(tiles_ptr + STAGES2 * STAGE2_BYTES + STAGING_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -615,8 +718,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   } else {
     // ===== epilogue (both CTAs): own 128 accumulator rows =====
     const int quarter = warp & 3;
-    uint32_t local = 0;
+    uint32_t local = 0, which = 0;
     bool alive = true;
+    const bool use_tma = !(p.accumulate != 0 && sizeof(OutT) == 2);
     for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters, ++local) {
       int m0, n0;
       decode_tile_pair(p, t, m0, n0);
@@ -626,29 +730,36 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const bool got = mbar_wait(smem_u32(&bars->acc_full[buf]), use & 1u, abort_flag, p.status);
       if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
-      const bool row_ok = row < static_cast<int>(p.Mo);
-      OutT* row_ptr = static_cast<OutT*>(p.C) + static_cast<int64_t>(row) * p.ldc;
       const uint32_t taddr = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(quarter * 32) << 16);
       const bool empty_k = p.Kc <= 0;
+      auto release = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->acc_empty[buf]), 0));
+      };
+      if (use_tma) {
+        epilogue_tile_tma<OutT>(&tmC, staging_base + static_cast<uint32_t>(warp - 2) * 8192u, which, taddr, m0 + quarter * 32, n0, 0,
+                                static_cast<int>(p.Mo), static_cast<int>(p.No), p.accumulate != 0, empty_k, lane, release);
+      } else {
+        const int row = m0 + quarter * 32 + lane;
+        const bool row_ok = row < static_cast<int>(p.Mo);
+        OutT* row_ptr = static_cast<OutT*>(p.C) + static_cast<int64_t>(row) * p.ldc;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t acc[32];
-        tmem_ld32(taddr + c * 32, acc);
-        tmem_ld_wait();
-        if (c == BN / 32 - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->acc_empty[buf]), 0));
-        }
-        if (empty_k) {
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+          if (c == BN / 32 - 1) release();
+          if (empty_k) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = 0u;
+            for (int j = 0; j < 32; ++j) acc[j] = 0u;
+          }
+          const int col0 = n0 + c * 32;
+          if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, true);
         }
-        const int col0 = n0 + c * 32;
-        if (row_ok && col0 < p.No) store_chunk32<OutT>(row_ptr, col0, static_cast<int>(p.No), acc, p.accumulate != 0);
       }
     }
+    if (lane == 0) bulk_wait_all();
   }
 
   // ===== teardown: nobody leaves while the partner may still touch this CTA's memory or barriers =====
@@ -692,40 +803,59 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D tensor map over the output for the epilogue's TMA stores: [groups, rows, cols] with a
+// box of 32 rows x 128 bytes, 128-byte swizzle. Plain outputs use groups = 1.
+bool make_map_c(CUtensorMap* map, void* base, int c_dtype, int64_t groups, int64_t rows, int64_t cols, int64_t ld,
+                int64_t group_stride) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  const cuuint64_t es = c_dtype == QF_DT_F32 ? 4 : 2;
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(groups)};
+  const cuuint64_t gs = groups > 1 ? static_cast<cuuint64_t>(group_stride) : static_cast<cuuint64_t>(rows) * static_cast<cuuint64_t>(ld);
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * es, gs * es};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / es), 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, c_dtype == QF_DT_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides,
+             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool A_MN, bool B_MN, typename OutT>
-cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid, cudaStream_t st) {
+cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
+                     cudaStream_t st) {
   auto kern = gemm_kernel<A_MN, B_MN, OutT>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, kp);
+  kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, tmC, kp);
   return cudaGetLastError();
 }
 
 template <bool A_MN, bool B_MN, typename OutT>
-cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid, cudaStream_t st) {
+cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
+                          cudaStream_t st) {
   auto kern = gemm_pair_kernel<A_MN, B_MN, OutT>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
   if (e != cudaSuccess) return e;
-  kern<<<grid, NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, kp);      // cluster shape (2,1,1) is a kernel attribute
+  kern<<<grid, NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);      // cluster shape (2,1,1) is a kernel attribute
   return cudaGetLastError();
 }
 
 template <typename OutT>
-cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid,
-                               cudaStream_t st) {
-  if (!a.a_mn_major && !a.b_mn_major) return launch_pair_t<false, false, OutT>(tmA, tmB, kp, grid, st);
-  if (!a.a_mn_major && a.b_mn_major) return launch_pair_t<false, true, OutT>(tmA, tmB, kp, grid, st);
-  if (a.a_mn_major && a.b_mn_major) return launch_pair_t<true, true, OutT>(tmA, tmB, kp, grid, st);
-  return launch_pair_t<true, false, OutT>(tmA, tmB, kp, grid, st);
+cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                               const KParams& kp, int grid, cudaStream_t st) {
+  if (!a.a_mn_major && !a.b_mn_major) return launch_pair_t<false, false, OutT>(tmA, tmB, tmC, kp, grid, st);
+  if (!a.a_mn_major && a.b_mn_major) return launch_pair_t<false, true, OutT>(tmA, tmB, tmC, kp, grid, st);
+  if (a.a_mn_major && a.b_mn_major) return launch_pair_t<true, true, OutT>(tmA, tmB, tmC, kp, grid, st);
+  return launch_pair_t<true, false, OutT>(tmA, tmB, tmC, kp, grid, st);
 }
 
 template <typename OutT>
-cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const KParams& kp, int grid,
-                          cudaStream_t st) {
-  if (!a.a_mn_major && !a.b_mn_major) return launch_t<false, false, OutT>(tmA, tmB, kp, grid, st);
-  if (!a.a_mn_major && a.b_mn_major) return launch_t<false, true, OutT>(tmA, tmB, kp, grid, st);
-  if (a.a_mn_major && a.b_mn_major) return launch_t<true, true, OutT>(tmA, tmB, kp, grid, st);
-  return launch_t<true, false, OutT>(tmA, tmB, kp, grid, st);
+cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                          const KParams& kp, int grid, cudaStream_t st) {
+  if (!a.a_mn_major && !a.b_mn_major) return launch_t<false, false, OutT>(tmA, tmB, tmC, kp, grid, st);
+  if (!a.a_mn_major && a.b_mn_major) return launch_t<false, true, OutT>(tmA, tmB, tmC, kp, grid, st);
+  if (a.a_mn_major && a.b_mn_major) return launch_t<true, true, OutT>(tmA, tmB, tmC, kp, grid, st);
+  return launch_t<true, false, OutT>(tmA, tmB, tmC, kp, grid, st);
 }
 
 }  // namespace
@@ -752,10 +882,12 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   if (a.b_mn_major) ok = make_map(&tmB, a.B, a.Kc, a.No, a.ldb, 64, BK);
   else ok = make_map(&tmB, a.B, a.No, a.Kc, a.ldb, BK, BN / 2);
   if (!ok) return cudaErrorInvalidValue;
+  CUtensorMap tmC;
+  if (!make_map_c(&tmC, a.C, a.c_dtype, 1, a.Mo, a.No, a.ldc, 0)) return cudaErrorInvalidValue;
   const int clusters = kp.num_tiles < kNumSMs / 2 ? kp.num_tiles : kNumSMs / 2;
   const int grid = 2 * clusters;
-  if (a.c_dtype == QF_DT_F32) return launch_pair_majors<float>(a, tmA, tmB, kp, grid, st);
-  return launch_pair_majors<__nv_bfloat16>(a, tmA, tmB, kp, grid, st);
+  if (a.c_dtype == QF_DT_F32) return launch_pair_majors<float>(a, tmA, tmB, tmC, kp, grid, st);
+  return launch_pair_majors<__nv_bfloat16>(a, tmA, tmB, tmC, kp, grid, st);
 }
 
 static int pair_mode() {
@@ -810,9 +942,12 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   }
   if (!ok) return cudaErrorInvalidValue;
 
+  CUtensorMap tmC;
+  const bool per_group_c = a.group_mode == 2;
+  if (!make_map_c(&tmC, a.C, a.c_dtype, per_group_c ? a.G : 1, kp.Mo, a.No, a.ldc, a.c_group_stride)) return cudaErrorInvalidValue;
   const int grid = kp.num_tiles < kNumSMs ? kp.num_tiles : kNumSMs;
-  if (a.c_dtype == QF_DT_F32) return launch_majors<float>(a, tmA, tmB, kp, grid, st);
-  return launch_majors<__nv_bfloat16>(a, tmA, tmB, kp, grid, st);
+  if (a.c_dtype == QF_DT_F32) return launch_majors<float>(a, tmA, tmB, tmC, kp, grid, st);
+  return launch_majors<__nv_bfloat16>(a, tmA, tmB, tmC, kp, grid, st);
 }
 
 }  // namespace qf
