@@ -64,6 +64,10 @@ typedef enum {
 #define QF_W_TSCALE_GIVEN 0x1u     /* linear calls: *w_tscale is an input (tied / shared scale)      */
 #define QF_A_TSCALE_GIVEN 0x2u     /* linear calls: *a_tscale is an input (running activation scale) */
 #define QF_ACCUMULATE_DW 0x4u      /* backward: dW += ... instead of dW = ... (gradient accumulation) */
+#define QF_FUSED_QDQ 0x8u          /* linear calls: quantize-dequantize MXFP4 operands inside the matmul kernel, on the
+                                      tiles staged in shared memory, instead of writing fake-quantized copies to the
+                                      workspace first. Same results bit for bit. Applies to MXFP4 operands of
+                                      non-grouped calls with M >= 256; anything else silently takes the default path. */
 
 const char* qf_status_string(qf_status_t s);
 int qf_version(void);
@@ -186,6 +190,11 @@ qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8
  * arrays) the quotient is compared bit for bit with the IEEE quotient; *mismatches (device u64)
  * receives the number of differences. */
 qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream);
+
+/* Self-test hook for the conversion-free MXFP4 rounding used inside the fused matmul kernel (packed BF16
+ * add/subtract of a magic constant): every BF16 bit pattern against every block-scale code in [8, 240]
+ * is compared with the conversion-instruction route; *mismatches (device u64) receives the count. */
+qf_status_t qf_selftest_mxfp4_bf16(uint64_t* mismatches, void* stream);
 
 #ifdef __cplusplus
 }

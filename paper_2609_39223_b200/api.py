@@ -16,7 +16,7 @@ FMT_NONE, FMT_NVFP4, FMT_MXFP4, FMT_Q4_K = 0, 1, 2, 3
 DT_BF16, DT_F32 = 0, 1
 OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 3, 4
 TENSOR_SCALE_GIVEN = 0x1
-W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW = 0x1, 0x2, 0x4
+W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ = 0x1, 0x2, 0x4, 0x8
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 
@@ -25,7 +25,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div", "qf_fq_linear_fwd_noalloc",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.qf_fq_linear_fwd_noalloc.restype = c_int
         L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
                                                c_void_p, c_void_p, c_uint32, c_void_p]
+        L.qf_selftest_mxfp4_bf16.restype = c_int
+        L.qf_selftest_mxfp4_bf16.argtypes = [c_void_p, c_void_p]
         L.qf_selftest_div.restype = c_int
         L.qf_selftest_div.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p]
         _lib = L
@@ -271,3 +273,10 @@ def qf_fq_linear_fwd_noalloc(X, W, Y, wq_fmt: int, aq_fmt: int, *, w_tscale=None
     _check(lib().qf_fq_linear_fwd_noalloc(_ptr(X), _ptr(W), _ptr(Y), _dt(Y.dtype), M, N, K, wq_fmt, aq_fmt, _ptr(w_tscale),
                                           _ptr(a_tscale), flags, _stream()), "qf_fq_linear_fwd_noalloc")
     return Y
+
+
+def qf_selftest_mxfp4_bf16() -> int:
+    """Mismatches between the conversion-free MXFP4 rounding and the conversion-instruction route (all inputs)."""
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(lib().qf_selftest_mxfp4_bf16(_ptr(out), _stream()), "qf_selftest_mxfp4_bf16")
+    return int(out.item())

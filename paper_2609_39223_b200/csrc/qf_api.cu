@@ -111,24 +111,8 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   if (M == 0 || N == 0) return QF_OK;
   Workspace w = carve(ws, N, K, groups);
   if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
-  const void* Wh = W;
-  const void* Xh = X;
-  if (K > 0) {
-    if (wq != QF_FMT_NONE) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
-      Wh = w.w_hat;
-    }
-    if (a_amax_out) {
-      if (cudaError_t e = launch_amax(X, M * K, w.header + 6, st)) return cu(e);
-      if (cudaError_t e = launch_amax_to_float(w.header + 6, a_amax_out, st)) return cu(e);
-    }
-    if (aq != QF_FMT_NONE) {
-      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
-      Xh = w.x_hat;
-    }
-  }
   GemmArgs g{};
-  g.A = Xh; g.B = Wh; g.C = Y;
+  g.C = Y;
   g.Mo = M; g.No = N; g.Kc = K;
   g.lda = K; g.ldb = K; g.ldc = N;
   g.a_mn_major = false; g.b_mn_major = false;
@@ -137,6 +121,26 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   if (grouped) {
     g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M;
   }
+  const bool may_fuse = (flags & QF_FUSED_QDQ) && gemm_can_fuse(g);
+  g.fuse_b_mxfp4 = may_fuse && wq == QF_FMT_MXFP4;
+  g.fuse_a_mxfp4 = may_fuse && aq == QF_FMT_MXFP4;
+  const void* Wh = W;
+  const void* Xh = X;
+  if (K > 0) {
+    if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      Wh = w.w_hat;
+    }
+    if (a_amax_out) {
+      if (cudaError_t e = launch_amax(X, M * K, w.header + 6, st)) return cu(e);
+      if (cudaError_t e = launch_amax_to_float(w.header + 6, a_amax_out, st)) return cu(e);
+    }
+    if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
+      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      Xh = w.x_hat;
+    }
+  }
+  g.A = Xh; g.B = Wh;
   return cu(launch_gemm(g, st));
 }
 
@@ -164,31 +168,28 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
   Workspace w = carve(ws, N, K, groups);
   if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
   if (dX) {
-    const void* Wh = W;
-    if (wq != QF_FMT_NONE) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
-      Wh = w.w_hat;
-    }
     // dX[M,K] = dY[M,N] . W_hat[N,K]: A = dY contraction-major, B = W_hat stored [contraction N, K]
     GemmArgs g{};
-    g.A = dY; g.B = Wh; g.C = dX;
+    g.A = dY; g.C = dX;
     g.Mo = M; g.No = K; g.Kc = N;
     g.lda = N; g.ldb = K; g.ldc = K;
     g.a_mn_major = false; g.b_mn_major = true;
     g.c_dtype = dx_dtype;
     g.status_word = w.header + kWsStatus;
     if (grouped) { g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M; }
+    g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && wq == QF_FMT_MXFP4 && gemm_can_fuse(g);
+    const void* Wh = W;
+    if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      Wh = w.w_hat;
+    }
+    g.B = Wh;
     if (cudaError_t e = launch_gemm(g, st)) return cu(e);
   }
   if (dW) {
-    const void* Xh = X;
-    if (aq != QF_FMT_NONE) {
-      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
-      Xh = w.x_hat;
-    }
     // dW[N,K] = dY[M,N]^T . X_hat[M,K]: both operands stored [contraction M, rows]
     GemmArgs g{};
-    g.A = dY; g.B = Xh; g.C = dW;
+    g.A = dY; g.C = dW;
     g.Mo = N; g.No = K; g.Kc = M;
     g.lda = N; g.ldb = K; g.ldc = K;
     g.a_mn_major = true; g.b_mn_major = true;
@@ -196,6 +197,13 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.accumulate = (flags & QF_ACCUMULATE_DW) != 0;
     g.status_word = w.header + kWsStatus;
     if (grouped) { g.group_mode = 2; g.group_offsets = offs; g.G = G; g.rows_padded = M; g.c_group_stride = N * K; }
+    g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && aq == QF_FMT_MXFP4 && gemm_can_fuse(g);
+    const void* Xh = X;
+    if (aq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
+      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      Xh = w.x_hat;
+    }
+    g.B = Xh;
     if (cudaError_t e = launch_gemm(g, st)) return cu(e);
   }
   return QF_OK;
@@ -389,6 +397,14 @@ qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_d
   if (qf_status_t s = noalloc_scratch_ptr(&scratch)) return s;
   return linear_fwd_impl(X, W, Y, y_dtype, nullptr, 1, M, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale, nullptr, flags, scratch,
                          QF_NOALLOC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
+}
+
+qf_status_t qf_selftest_mxfp4_bf16(uint64_t* mismatches, void* stream) {
+  if (!mismatches) return QF_ERR_NULL;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaError_t e = cudaMemsetAsync(mismatches, 0, 8, st)) return cu(e);
+  return cu(launch_selftest_mxfp4_bf16(reinterpret_cast<unsigned long long*>(mismatches), st));
 }
 
 qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream) {

@@ -77,6 +77,48 @@ __device__ __forceinline__ uint32_t mxfp4_scale_code(uint32_t amax_bf16_bits) {
   return static_cast<uint32_t>(max(e - 2, 0));
 }
 
+__device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
+__device__ __forceinline__ uint32_t bf2_bits(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
+__device__ __forceinline__ __nv_bfloat162 bits_bf2(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
+
+// max |x| over the 8 BF16 values of one 16-byte chunk, as BF16 bits (sign clear)
+__device__ __forceinline__ uint32_t chunk8_amax_bits(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+  const __nv_bfloat162 a = __hmax2(__habs2(bits_bf2(w0)), __habs2(bits_bf2(w1)));
+  const __nv_bfloat162 b = __hmax2(__habs2(bits_bf2(w2)), __habs2(bits_bf2(w3)));
+  const uint32_t m = bf2_bits(__hmax2(a, b));
+  return max(m & 0xFFFFu, m >> 16);
+}
+
+// MXFP4 quantize-dequantize of one packed BF16 pair given its block's max |x| (BF16 bits):
+// x_hat = 2^p * E2M1(x * 2^-p), p = floor(log2 amax) - 2 (Eq. mxfp4-dequant). Every product is exact.
+__device__ __forceinline__ uint32_t mxfp4_qdq_pair(uint32_t w, float2 inv, float2 sc, uint32_t keep) {
+  const float2 v = __fmul2_rn(unpack2(w), inv);
+  const uint32_t byte = e2m1x2_encode(v.x, v.y) & keep;
+  const float2 o = __fmul2_rn(e2m1x2_decode(byte), sc);
+  return pack_bf16x2(o.x, o.y);
+}
+
+// The same MXFP4 rounding done entirely in packed BF16 arithmetic (no format conversions, which run
+// on a narrow pipe): for |x| in the binade [2^e, 2^(e+1)) the E2M1 grid scaled by 2^p has spacing
+// 2^(e-1) (one mantissa bit), and below 2^p it has the spacing of the first binade, 2^(p-1). Adding
+// and subtracting 1.5 * 2^(e+6) in BF16 (8 significant bits) therefore rounds |x| to that spacing with
+// round-to-nearest-even, and "even multiple of the spacing" coincides with "even E2M1 code"; the
+// result is then clamped to 6 * 2^p and the sign of x restored. `one2` is 2^p and `six2` 6 * 2^p as
+// packed BF16 pairs. Valid while all of these are normal BF16 numbers: scale code in [8, 240].
+__device__ __forceinline__ bool mxfp4_bf16_path_ok(uint32_t scale_code) { return scale_code >= 8u && scale_code <= 240u; }
+__device__ __forceinline__ uint32_t mxfp4_one2(uint32_t scale_code) { return (scale_code << 7) | (scale_code << 23); }
+__device__ __forceinline__ uint32_t mxfp4_six2(uint32_t scale_code) { return mxfp4_one2(scale_code + 2u) | 0x00400040u; }
+__device__ __forceinline__ uint32_t mxfp4_qdq_pair_bf16(uint32_t w, uint32_t one2, uint32_t six2) {
+  const uint32_t a = w & 0x7FFF7FFFu;
+  const uint32_t t = bf2_bits(__hmax2(bits_bf2(a), bits_bf2(one2)));
+  const uint32_t magic = (t & 0x7F807F80u) + 0x03400340u;            // 1.5 * 2^(e+6) per lane
+  __nv_bfloat162 r = __hadd2(bits_bf2(a), bits_bf2(magic));           // one rounding: nearest multiple of the spacing
+  r = __hsub2(r, bits_bf2(magic));                                    // exact
+  r = __hmin2(r, bits_bf2(six2));
+  return bf2_bits(r) | (w & 0x80008000u);
+}
+
 // ---- host-side launchers implemented in the .cu files ---------------------------------------
 
 struct QdqArgs {
@@ -100,6 +142,7 @@ cudaError_t launch_dequant(int fmt, const void* codes, const void* scales, const
                            int64_t cols, void* out, cudaStream_t st);
 cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,
                                 cudaStream_t st);
+cudaError_t launch_selftest_mxfp4_bf16(unsigned long long* mismatches, cudaStream_t st);
 cudaError_t launch_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1, uint8_t* e4m3, cudaStream_t st);
 
 // C[Mo, No] (+)= sum_c A(m, c) * B(n, c). Operand storage: K-major = [rows, contraction] row-major,
@@ -123,8 +166,10 @@ struct GemmArgs {
   int64_t c_group_stride;        // elements between consecutive groups of C (mode 2)
   int64_t rows_padded;           // mode 1: total rows of A / C; mode 2: total contraction rows
   uint32_t* status_word;         // device word receiving QF_ERR_TIMEOUT if a wait expires
+  bool fuse_a_mxfp4, fuse_b_mxfp4;   // apply the MXFP4 quantize-dequantize to the staged tiles inside the kernel
 };
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+bool gemm_can_fuse(const GemmArgs& a);
 
 }  // namespace qf

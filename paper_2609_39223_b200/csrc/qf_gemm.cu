@@ -539,8 +539,14 @@ constexpr int B2_BYTES = (BN / 2) * BK * 2;     // 16 KB: this CTA's 128 rows of
 constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256;
 
+constexpr int TRANSFORM_WARPS = 8;                       // fused variant: warps that quantize-dequantize staged tiles
+constexpr int TRANSFORM_GROUPS = 4;                      // group g takes k-blocks g, g + 4, ...
+constexpr int WARPS_PER_GROUP = TRANSFORM_WARPS / TRANSFORM_GROUPS;
+constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * TRANSFORM_WARPS;
+
 struct alignas(8) Barriers2 {
-  uint64_t full[STAGES2];       // leader's copy is the live one
+  uint64_t ready[STAGES2];      // fused variant, leader's copy: both CTAs' tiles have been quantized in place
+  uint64_t full[STAGES2];       // leader's copy is the live one (fused variant: each CTA's own copy)
   uint64_t empty[STAGES2];      // one per CTA, released by the leader's commit multicast
   uint64_t acc_full[2];         // one per CTA, published by the leader's commit multicast
   uint64_t acc_empty[2];        // leader's copy is the live one: 8 arrivals (4 epilogue warps x 2 CTAs)
@@ -610,8 +616,68 @@ __device__ __forceinline__ void decode_tile_pair(const KParams& p, int t, int& m
   n0 = (within / rows_in_band) * BN;
 }
 
-template <bool A_MN, bool B_MN, typename OutT>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
+// In-place MXFP4 quantize-dequantize of `nchunks` 16-byte chunks of a staged operand tile by the 256
+// transform threads. A tile is a stack of 128-byte rows holding 64 consecutive elements of the
+// tensor's last (block) dimension, whatever the operand's majorness, so a 32-element block is an aligned
+// group of four chunks; the 128-byte swizzle permutes chunks only inside aligned groups of eight by
+// an XOR, which maps aligned groups of four onto aligned groups of four. Lane l takes chunk l of each
+// 512-byte span (bank-conflict free); the four lanes of a block combine their maxima by shuffles.
+// One batch: PER chunks per lane, loads first, then shuffles, then independent arithmetic chains, then stores.
+template <int PER>
+__device__ __forceinline__ void mxfp4_transform_batch(uint32_t slab) {
+  uint4 v[PER];
+  uint32_t m[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) v[i] = ld_shared_v4(slab + static_cast<uint32_t>(i) * 512u);
+#pragma unroll
+  for (int i = 0; i < PER; ++i) m[i] = chunk8_amax_bits(v[i].x, v[i].y, v[i].z, v[i].w);
+#pragma unroll
+  for (int i = 0; i < PER; ++i) m[i] = max(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], 1));
+#pragma unroll
+  for (int i = 0; i < PER; ++i) m[i] = max(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], 2));
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const uint32_t code = mxfp4_scale_code(m[i]);
+    const uint32_t dst = slab + static_cast<uint32_t>(i) * 512u;
+    if (mxfp4_bf16_path_ok(code)) {
+      // conversion-free rounding in packed BF16 arithmetic (the common case)
+      const uint32_t one2 = mxfp4_one2(code), six2 = mxfp4_six2(code);
+      st_shared_v4(dst, mxfp4_qdq_pair_bf16(v[i].x, one2, six2), mxfp4_qdq_pair_bf16(v[i].y, one2, six2),
+                   mxfp4_qdq_pair_bf16(v[i].z, one2, six2), mxfp4_qdq_pair_bf16(v[i].w, one2, six2));
+    } else {
+      // all-zero blocks (tile padding) and blocks at the very ends of the BF16 exponent range
+      const float2 inv = splat(e8m0_inv_scale(code)), sc = splat(e8m0_scale(code));
+      const uint32_t keep = m[i] == 0 ? 0u : 0xFFu;
+      st_shared_v4(dst, mxfp4_qdq_pair(v[i].x, inv, sc, keep), mxfp4_qdq_pair(v[i].y, inv, sc, keep),
+                   mxfp4_qdq_pair(v[i].z, inv, sc, keep), mxfp4_qdq_pair(v[i].w, inv, sc, keep));
+    }
+  }
+}
+
+// A staged tile of NCHUNKS 16-byte chunks, split between the WARPS_PER_GROUP warps of one transform group:
+// each warp owns a contiguous slab and walks it in batches of four chunks per lane (512 bytes per warp
+// per load instruction: bank-conflict free, and every aligned group of four lanes holds one 32-element block).
+template <int NCHUNKS>
+__device__ __forceinline__ void mxfp4_transform_tile(uint32_t base, int warp_in_group, int lane) {
+  constexpr int PER_WARP = NCHUNKS / WARPS_PER_GROUP;          // chunks per warp
+  constexpr int BATCH = 4;
+  static_assert(PER_WARP % (32 * BATCH) == 0, "tile must split evenly");
+  const uint32_t slab = base + static_cast<uint32_t>(warp_in_group * PER_WARP + lane) * 16u;
+#pragma unroll 1
+  for (int b = 0; b < PER_WARP / (32 * BATCH); ++b) mxfp4_transform_batch<BATCH>(slab + static_cast<uint32_t>(b) * (32u * BATCH * 16u));
+}
+
+// FUSE: bit 0 = quantize-dequantize the staged A tile (MXFP4), bit 1 = the staged B tile. With FUSE != 0
+// eight extra warps transform each stage in shared memory between the TMA arrival and the MMA issue, so
+// the fake-quantized operand never exists in global memory.
+template <bool A_MN, bool B_MN, typename OutT, int FUSE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FUSE ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -631,6 +697,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) {
+      mbar_init(smem_u32(&bars->ready[s]), 2 * WARPS_PER_GROUP);
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
@@ -662,10 +729,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status)) { alive = false; break; }
           const uint32_t full_local = smem_u32(&bars->full[stage]);
-          const uint32_t full_leader = mapa_shared(full_local, 0);
+          // plain variant: both CTAs' bytes are counted on the leader's barrier, which the MMA thread watches;
+          // fused variant: each CTA counts its own bytes, its transform warps watch its own barrier
+          const uint32_t full_leader = FUSE ? full_local : mapa_shared(full_local, 0);
           const uint32_t a_dst = tiles_base + stage * STAGE2_BYTES;
           const uint32_t b_dst = a_dst + A2_BYTES;
-          if (leader) mbar_expect_tx(full_local, 2 * STAGE2_BYTES);      // both CTAs' bytes land on this barrier
+          if (FUSE) mbar_expect_tx(full_local, STAGE2_BYTES);
+          else if (leader) mbar_expect_tx(full_local, 2 * STAGE2_BYTES);
           if (A_MN) {
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * 8192, &tmA, m0 + 64 * i, k, full_leader);
@@ -698,7 +768,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
         uint32_t accumulate = 0;
         for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
-          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status)) { alive = false; break; }
+          if (!mbar_wait(smem_u32(FUSE ? &bars->ready[stage] : &bars->full[stage]), phase, abort_flag, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
           const uint64_t a_desc = smem_desc<A_MN>(a_addr);
@@ -713,6 +783,31 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         if (!alive) break;
         umma_commit_pair(smem_u32(&bars->acc_full[buf]));
+      }
+    }
+  } else if (FUSE && warp >= 6) {
+    // ===== transform warps (both CTAs): MXFP4 quantize-dequantize of the staged tiles, in place =====
+    // Group g handles k-blocks g, g + GROUPS, ...: the groups work on different stages at the same time,
+    // so the wake-up / fence / signal latency of one stage overlaps the arithmetic of the others.
+    const int twarp = warp - 6;
+    const int group = twarp / WARPS_PER_GROUP, wig = twarp % WARPS_PER_GROUP;
+    uint32_t it = 0;                                  // running k-block count over all of this CTA's tiles
+    bool alive = true;
+    for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters) {
+      for (int k = 0; k < static_cast<int>(p.Kc); k += BK, ++it) {
+        if (static_cast<int>(it % TRANSFORM_GROUPS) != group) continue;
+        const uint32_t stage = it % STAGES2, phase = (it / STAGES2) & 1u;
+        // one lane polls the barrier; the warp then proceeds together (the shuffles need all lanes)
+        int got = 1;
+        if (lane == 0) got = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status) ? 1 : 0;
+        got = __shfl_sync(0xFFFFFFFFu, got, 0);
+        if (!got) { alive = false; break; }
+        const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
+        if (FUSE & 1) mxfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane);
+        if (FUSE & 2) mxfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane);
+        fence_async_smem();                          // make the generic-proxy writes visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->ready[stage]), 0));
       }
     }
   } else {
@@ -830,23 +925,38 @@ cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUten
   return cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN, typename OutT>
+template <bool A_MN, bool B_MN, typename OutT, int FUSE>
 cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
                           cudaStream_t st) {
-  auto kern = gemm_pair_kernel<A_MN, B_MN, OutT>;
+  auto kern = gemm_pair_kernel<A_MN, B_MN, OutT, FUSE>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
   if (e != cudaSuccess) return e;
-  kern<<<grid, NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);      // cluster shape (2,1,1) is a kernel attribute
+  kern<<<grid, FUSE ? NUM_THREADS_FUSED : NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);   // cluster shape (2,1,1) is a kernel attribute
   return cudaGetLastError();
 }
 
 template <typename OutT>
 cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
                                const KParams& kp, int grid, cudaStream_t st) {
-  if (!a.a_mn_major && !a.b_mn_major) return launch_pair_t<false, false, OutT>(tmA, tmB, tmC, kp, grid, st);
-  if (!a.a_mn_major && a.b_mn_major) return launch_pair_t<false, true, OutT>(tmA, tmB, tmC, kp, grid, st);
-  if (a.a_mn_major && a.b_mn_major) return launch_pair_t<true, true, OutT>(tmA, tmB, tmC, kp, grid, st);
-  return launch_pair_t<true, false, OutT>(tmA, tmB, tmC, kp, grid, st);
+  const int fuse = (a.fuse_a_mxfp4 ? 1 : 0) | (a.fuse_b_mxfp4 ? 2 : 0);
+  if (!a.a_mn_major && !a.b_mn_major) {
+    if (fuse == 3) return launch_pair_t<false, false, OutT, 3>(tmA, tmB, tmC, kp, grid, st);
+    if (fuse == 2) return launch_pair_t<false, false, OutT, 2>(tmA, tmB, tmC, kp, grid, st);
+    if (fuse == 1) return launch_pair_t<false, false, OutT, 1>(tmA, tmB, tmC, kp, grid, st);
+    return launch_pair_t<false, false, OutT, 0>(tmA, tmB, tmC, kp, grid, st);
+  }
+  if (!a.a_mn_major && a.b_mn_major) {
+    if (fuse == 2) return launch_pair_t<false, true, OutT, 2>(tmA, tmB, tmC, kp, grid, st);
+    if (fuse != 0) return cudaErrorInvalidValue;
+    return launch_pair_t<false, true, OutT, 0>(tmA, tmB, tmC, kp, grid, st);
+  }
+  if (a.a_mn_major && a.b_mn_major) {
+    if (fuse == 2) return launch_pair_t<true, true, OutT, 2>(tmA, tmB, tmC, kp, grid, st);
+    if (fuse != 0) return cudaErrorInvalidValue;
+    return launch_pair_t<true, true, OutT, 0>(tmA, tmB, tmC, kp, grid, st);
+  }
+  if (fuse != 0) return cudaErrorInvalidValue;
+  return launch_pair_t<true, false, OutT, 0>(tmA, tmB, tmC, kp, grid, st);
 }
 
 template <typename OutT>
@@ -900,9 +1010,13 @@ static int pair_mode() {
   return mode;
 }
 
+// True if launch_gemm would run this problem on the kernel that can quantize-dequantize staged tiles itself.
+bool gemm_can_fuse(const GemmArgs& a) { return a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode() != 0; }
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
   if (a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode()) return launch_gemm_pair(a, st);
+  if (a.fuse_a_mxfp4 || a.fuse_b_mxfp4) return cudaErrorInvalidValue;       // only the two-CTA kernel fuses (see gemm_can_fuse)
   KParams kp{};
   kp.C = a.C;
   kp.Mo = a.Mo;

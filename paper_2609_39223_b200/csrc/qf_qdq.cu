@@ -72,7 +72,6 @@ __global__ void amax_to_float_kernel(const uint32_t* amax_bits, float* out) { *o
 #define QF_DIV_STEPS 1      // residual corrections after the first product (1 suffices with an exact reciprocal)
 #endif
 
-__device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
 
 __device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
   const float2 ny = splat(-y), r = splat(rc);
@@ -98,10 +97,7 @@ __device__ __forceinline__ float copysign_bits(float mag, float sgn) {
   return __uint_as_float((__float_as_uint(mag) & 0x7FFFFFFFu) | (__float_as_uint(sgn) & 0x80000000u));
 }
 
-__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
 
-__device__ __forceinline__ uint32_t bf2_bits(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
-__device__ __forceinline__ __nv_bfloat162 bits_bf2(uint32_t v) { return *reinterpret_cast<__nv_bfloat162*>(&v); }
 
 // max |x| over 16 BF16 values held in 8 words, as BF16 bits (sign clear)
 __device__ __forceinline__ uint32_t unit_amax_bits(const uint32_t (&w)[8]) {
@@ -500,6 +496,24 @@ __global__ void selftest_cvt_kernel(const float* __restrict__ in, int64_t n, uin
   if (e4m3) e4m3[i] = static_cast<uint8_t>(e4m3_encode(fabsf(x)));
 }
 
+// every BF16 bit pattern x against every scale code the packed-BF16 MXFP4 rounding is used for:
+// it must give the same BF16 result as the conversion-instruction route
+__global__ void selftest_mxfp4_bf16_kernel(unsigned long long* __restrict__ mismatches) {
+  const uint32_t code = 8u + blockIdx.x;                    // grid = 233 blocks: codes 8 .. 240
+  const float2 inv = splat(e8m0_inv_scale(code)), sc = splat(e8m0_scale(code));
+  const uint32_t one2 = mxfp4_one2(code), six2 = mxfp4_six2(code);
+  const uint32_t amax_hi = ((code + 2u) << 7) | 0x7Fu;      // the largest |x| a block with this scale can hold
+  unsigned long long bad = 0;
+  for (uint32_t x = threadIdx.x; x < 0x10000u; x += blockDim.x) {
+    if ((x & 0x7FFFu) > amax_hi) continue;
+    const uint32_t w = x | (((x * 40503u) & 0xFFFFu) << 16);  // pair it with another pattern in the high half
+    const uint32_t hi = (w >> 16) & 0x7FFFu;
+    const uint32_t w2 = hi > amax_hi ? (w & 0xFFFFu) : w;
+    if (mxfp4_qdq_pair(w2, inv, sc, 0xFFu) != mxfp4_qdq_pair_bf16(w2, one2, six2)) ++bad;
+  }
+  if (bad) atomicAdd(mismatches, bad);
+}
+
 int grid_for(int64_t nchunks, int per_thread) {
   int64_t blocks = (nchunks + static_cast<int64_t>(kThreads) * per_thread - 1) / (static_cast<int64_t>(kThreads) * per_thread);
   const int64_t cap = static_cast<int64_t>(kNumSMs) * 8;       // 8 resident blocks of 256 threads per SM
@@ -574,6 +588,11 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
   q.tscale_in = nullptr;
   q.reverse = true;
   return launch_qdq(q, st);
+}
+
+cudaError_t launch_selftest_mxfp4_bf16(unsigned long long* mismatches, cudaStream_t st) {
+  selftest_mxfp4_bf16_kernel<<<233, 256, 0, st>>>(mismatches);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,

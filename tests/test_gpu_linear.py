@@ -226,3 +226,23 @@ def test_full_size_moe_grouped_mxfp4_sampled_experts():
         dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, fmt, fmt)
         _close(dx[a:b], dx_ref, f"expert {g} dX")
         _close(dw[g], dw_ref, f"expert {g} dW")
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_MXFP4, api.FMT_NONE), (api.FMT_NONE, api.FMT_MXFP4),
+                                   (api.FMT_MXFP4, api.FMT_NVFP4)])
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (520, 776, 1024), (1024, 1024, 2048)])
+def test_in_kernel_mxfp4_quantization_is_bitwise_the_workspace_path(wq, aq, M, N, K):
+    """QF_FUSED_QDQ quantizes the staged shared-memory tiles inside the matmul kernel. The operands it
+    produces are the same bits as the materialised copies, and the accumulation order is the same, so
+    every output must be identical to the default path's, not merely close."""
+    c = synth.linear_case(M, N, K, seed=M + K, outlier_channels=4)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    y0 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32)
+    dx0, dw0 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    y1 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32, flags=api.FUSED_QDQ, ws=ws)
+    dx1, dw1 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, flags=api.FUSED_QDQ, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+    # and against the oracle, like every other path
+    _close(y1, oracle.fq_linear_fwd(torch_to_bits(c.X), torch_to_bits(c.W), wq, aq), "Y fused")

@@ -201,3 +201,7 @@ def test_large_ragged_tensor_stays_inside_its_buffers(fmt, name):
         for raw in (raw_o, raw_c, raw_s):
             assert bool((raw[:pad] == 0xA5).all()) and bool((raw[-pad:] == 0xA5).all())
         np.testing.assert_array_equal(torch_to_bits(out), o["out"])
+
+
+def test_conversion_free_mxfp4_rounding_matches_the_conversion_route_exhaustively():
+    assert api.qf_selftest_mxfp4_bf16() == 0
