@@ -457,7 +457,10 @@ def run_ours(args):
             "e2e": e2e,
             "gpu_launches": KERNELS_PER_STEP * args.steps,
             "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel (tcgen05 cta_group::2 BF16, 256x256x64 tiles per CTA pair)", "achieved": achieved,
-                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
+                         # mean dram__bytes_read.sum + dram__bytes_write.sum per launch over the three matmuls of a
+                         # step, from the full-size ncu capture summarised in profiles/gemm_pair_kernel_mxfp4_linear.md
+                         "traffic": 916.2e6 if (M, N, K) == (8192, 12288, 4096) else None,
                          "peak_source": f"{peaks['source']} cuBLAS bf16 burst", "ms_per_launch": gemm_ms,
                          "frac_of_sustained": achieved / peaks["bf16_sustained"] if achieved else None,
                          "frac_of_2250_datasheet": achieved / 2250.0 if achieved else None,

@@ -55,6 +55,7 @@ struct KParams {
   int64_t Mo, No, Kc, ldc;
   int c_dtype, accumulate;
   int tiles_m, tiles_n, num_tiles;
+  int band;                  // row-tiles per rasterization band (see band_rows())
   int group_mode, G;
   const int32_t* offs;
   int64_t b_group_rows;      // mode 1: rows one group occupies in B's 2-D tensor map
@@ -195,11 +196,11 @@ __device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_g
     g = t / per;
     t -= g * per;
   }
-  // m fastest inside bands of 8 row-tiles: concurrently running CTAs share A and B tiles in L2
-  const int band = 8 * p.tiles_n;
+  // m fastest inside bands of p.band row-tiles: concurrently running CTAs share A and B tiles in L2
+  const int band = p.band * p.tiles_n;
   const int bidx = t / band;
-  const int first_m = bidx * 8;
-  const int rows_in_band = min(8, p.tiles_m - first_m);
+  const int first_m = bidx * p.band;
+  const int rows_in_band = min(p.band, p.tiles_m - first_m);
   const int within = t - bidx * band;
   r.m0 = (first_m + within % rows_in_band) * BM;
   r.n0 = (within / rows_in_band) * BN;
@@ -607,10 +608,10 @@ __device__ __forceinline__ uint32_t instr_desc_pair() {
 }
 
 __device__ __forceinline__ void decode_tile_pair(const KParams& p, int t, int& m0, int& n0) {
-  const int band = 8 * p.tiles_n;
+  const int band = p.band * p.tiles_n;
   const int bidx = t / band;
-  const int first_m = bidx * 8;
-  const int rows_in_band = min(8, p.tiles_m - first_m);
+  const int first_m = bidx * p.band;
+  const int rows_in_band = min(p.band, p.tiles_m - first_m);
   const int within = t - bidx * band;
   m0 = (first_m + within % rows_in_band) * (2 * BM);
   n0 = (within / rows_in_band) * BN;
@@ -898,6 +899,18 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-tiles per rasterization band. Tiles are walked row-tile fastest inside a band, so the band's A
+// panel (band * tile_rows * Kc BF16 values) is what must stay in the 126 MB L2 while B streams past once
+// per band: the larger the band the fewer times B is re-read from HBM. The panel is kept near 40 MB.
+int band_rows(int64_t tile_rows, int64_t Kc, int tiles_m) {
+  const int64_t per_tile = tile_rows * (Kc > 0 ? Kc : 1) * 2;
+  int64_t band = (40ll << 20) / per_tile;
+  if (band < 4) band = 4;
+  if (band > 32) band = 32;
+  if (band > tiles_m) band = tiles_m;
+  return static_cast<int>(band < 1 ? 1 : band);
+}
+
 // 3-D tensor map over the output for the epilogue's TMA stores: [groups, rows, cols] with a
 // box of 32 rows x 128 bytes, 128-byte swizzle. Plain outputs use groups = 1.
 bool make_map_c(CUtensorMap* map, void* base, int c_dtype, int64_t groups, int64_t rows, int64_t cols, int64_t ld,
@@ -984,6 +997,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.tiles_m = static_cast<int>((a.Mo + 2 * BM - 1) / (2 * BM));
   kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
   kp.num_tiles = kp.tiles_m * kp.tiles_n;
+  kp.band = band_rows(2 * BM, a.Kc, kp.tiles_m);
   CUtensorMap tmA, tmB;
   bool ok;
   if (a.a_mn_major) ok = make_map(&tmA, a.A, a.Kc, a.Mo, a.lda, 64, BK);
@@ -1034,6 +1048,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   kp.tiles_m = static_cast<int>((a_rows_total + BM - 1) / BM);
   kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
   kp.num_tiles = kp.tiles_m * kp.tiles_n * (a.group_mode == 2 ? a.G : 1);
+  kp.band = band_rows(BM, a.group_mode == 2 ? a.rows_padded / (a.G > 0 ? a.G : 1) : a.Kc, kp.tiles_m);
   if (a.group_mode == 1) kp.Mo = a.rows_padded;
   if (kp.num_tiles <= 0) return cudaSuccess;
 
