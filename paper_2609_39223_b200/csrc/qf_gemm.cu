@@ -535,10 +535,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // =====================================================================================================
 
 constexpr int STAGES2 = 6;
+constexpr int MAX_PAIR_GROUPS = 256;     // experts the two-CTA kernel's shared-memory tile table holds
 constexpr int A2_BYTES = BM * BK * 2;           // 16 KB: this CTA's 128 rows of A
 constexpr int B2_BYTES = (BN / 2) * BK * 2;     // 16 KB: this CTA's 128 rows of B
 constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256 + 4 * (MAX_PAIR_GROUPS + 4);
 
 constexpr int TRANSFORM_WARPS = 8;                       // fused variant: warps that quantize-dequantize staged tiles
 constexpr int TRANSFORM_GROUPS = 4;                      // group g takes k-blocks g, g + 4, ...
@@ -553,6 +554,7 @@ struct alignas(8) Barriers2 {
   uint64_t acc_empty[2];        // leader's copy is the live one: 8 arrivals (4 epilogue warps x 2 CTAs)
   uint32_t tmem_base;
   int abort_flag;
+  int cum[MAX_PAIR_GROUPS + 1];  // grouped mode 1: pair row-tiles before each expert (prefix sum)
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -607,14 +609,54 @@ __device__ __forceinline__ uint32_t instr_desc_pair() {
          (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>((2 * BM) >> 4) << 24);
 }
 
-__device__ __forceinline__ void decode_tile_pair(const KParams& p, int t, int& m0, int& n0) {
+struct PairTile {
+  int m0, n0;            // first output row / column of the 256 x 256 pair tile
+  int k_begin, k_end;    // contraction range
+  int b_row_off;         // mode 1: row offset of this tile's expert in B's 2-D tensor map
+  int z;                 // mode 2: which per-expert output matrix
+  int rows_limit;        // output rows at or beyond this index do not belong to this tile's matrix / segment
+};
+
+// Pair tiles are walked row-tile fastest inside bands (see band_rows()). Grouped mode 1: the row-tile
+// index counts 256-row tiles expert by expert (cum[] = tiles before each expert, built at kernel start);
+// a segment with an odd number of 128-row blocks ends in a tile whose second half lies in the next
+// expert's rows: that half is computed and thrown away (rows_limit = end of the segment).
+__device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum, int tiles_m, int t) {
+  PairTile r;
+  r.k_begin = 0;
+  r.k_end = static_cast<int>(p.Kc);
+  r.b_row_off = 0;
+  r.z = 0;
+  r.rows_limit = static_cast<int>(p.Mo);
+  int g = 0;
+  if (p.group_mode == 2) {
+    const int per = tiles_m * p.tiles_n;
+    g = t / per;
+    t -= g * per;
+  }
   const int band = p.band * p.tiles_n;
   const int bidx = t / band;
   const int first_m = bidx * p.band;
-  const int rows_in_band = min(p.band, p.tiles_m - first_m);
+  const int rows_in_band = min(p.band, tiles_m - first_m);
   const int within = t - bidx * band;
-  m0 = (first_m + within % rows_in_band) * (2 * BM);
-  n0 = (within / rows_in_band) * BN;
+  const int mt = first_m + within % rows_in_band;
+  r.n0 = (within / rows_in_band) * BN;
+  r.m0 = mt * (2 * BM);
+  if (p.group_mode == 1) {
+    int lo = 0, hi = p.G;                     // invariant: cum[lo] <= mt < cum[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (cum[mid] <= mt) lo = mid; else hi = mid;
+    }
+    r.m0 = __ldg(p.offs + lo) + (mt - cum[lo]) * (2 * BM);
+    r.rows_limit = __ldg(p.offs + lo + 1);
+    r.b_row_off = lo * static_cast<int>(p.b_group_rows);
+  } else if (p.group_mode == 2) {
+    r.k_begin = __ldg(p.offs + g);
+    r.k_end = __ldg(p.offs + g + 1);
+    r.z = g;
+  }
+  return r;
 }
 
 __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
@@ -711,23 +753,49 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(&bars->tmem_base), TMEM_COLS);
+  if (warp == 2 && p.group_mode == 1) {
+    // prefix sum of pair row-tiles per expert (G <= MAX_PAIR_GROUPS): lane l takes experts 8l .. 8l+7
+    int cnt[8], sum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int g = lane * 8 + j;
+      cnt[j] = g < p.G ? (__ldg(p.offs + g + 1) - __ldg(p.offs + g) + 2 * BM - 1) / (2 * BM) : 0;
+      sum += cnt[j];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= d) incl += up;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int g = lane * 8 + j;
+      if (g <= p.G) bars->cum[g] = run;
+      run += cnt[j];
+    }
+    if (lane * 8 + 8 == p.G) bars->cum[p.G] = run;      // G a multiple of 8: the total has no lane of its own when G = 256
+  }
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();                               // both CTAs' barriers exist before any remote access
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  const int* cum = bars->cum;
+  const int tiles_m = p.group_mode == 1 ? cum[p.G] : p.tiles_m;
+  const int num_tiles = p.group_mode == 1 ? tiles_m * p.tiles_n : p.num_tiles;
 
   if (warp == 0) {
     // ===== TMA producer (both CTAs): own rows of A, own half of B, counted on the leader's barrier =====
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued = 0;
       bool alive = true;
-      for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters) {
-        int m0, n0;
-        decode_tile_pair(p, t, m0, n0);
-        m0 += static_cast<int>(rank) * BM;
-        n0 += static_cast<int>(rank) * (BN / 2);
-        for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
+      for (int t = cluster_id; t < num_tiles && alive; t += num_clusters) {
+        const PairTile tile = decode_pair(p, cum, tiles_m, t);
+        const int m0 = tile.m0 + static_cast<int>(rank) * BM;
+        const int n0 = tile.n0 + static_cast<int>(rank) * (BN / 2);
+        for (int k = tile.k_begin; k < tile.k_end; k += BK) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status)) { alive = false; break; }
           const uint32_t full_local = smem_u32(&bars->full[stage]);
           // plain variant: both CTAs' bytes are counted on the leader's barrier, which the MMA thread watches;
@@ -745,9 +813,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
           if (B_MN) {
 #pragma unroll
-            for (int i = 0; i < BN / 2 / 64; ++i) tma_load_2d_pair(b_dst + i * 8192, &tmB, n0 + 64 * i, k, full_leader);
+            for (int i = 0; i < BN / 2 / 64; ++i) tma_load_2d_pair(b_dst + i * 8192, &tmB, n0 + 64 * i, tile.b_row_off + k, full_leader);
           } else {
-            tma_load_2d_pair(b_dst, &tmB, k, n0, full_leader);
+            tma_load_2d_pair(b_dst, &tmB, k, tile.b_row_off + n0, full_leader);
           }
           ++issued;
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
@@ -761,14 +829,15 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint32_t idesc = instr_desc_pair<A_MN, B_MN>();
       uint32_t stage = 0, phase = 0, local = 0;
       bool alive = true;
-      for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters, ++local) {
+      for (int t = cluster_id; t < num_tiles && alive; t += num_clusters, ++local) {
+        const PairTile tile = decode_pair(p, cum, tiles_m, t);
         const uint32_t buf = local & 1u;
         const uint32_t use = local >> 1;
         if (!mbar_wait(smem_u32(&bars->acc_empty[buf]), (use & 1u) ^ 1u, abort_flag, p.status)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
         uint32_t accumulate = 0;
-        for (int k = 0; k < static_cast<int>(p.Kc); k += BK) {
+        for (int k = tile.k_begin; k < tile.k_end; k += BK) {
           if (!mbar_wait(smem_u32(FUSE ? &bars->ready[stage] : &bars->full[stage]), phase, abort_flag, p.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
@@ -794,8 +863,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int group = twarp / WARPS_PER_GROUP, wig = twarp % WARPS_PER_GROUP;
     uint32_t it = 0;                                  // running k-block count over all of this CTA's tiles
     bool alive = true;
-    for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters) {
-      for (int k = 0; k < static_cast<int>(p.Kc); k += BK, ++it) {
+    for (int t = cluster_id; t < num_tiles && alive; t += num_clusters) {
+      const PairTile tile = decode_pair(p, cum, tiles_m, t);
+      for (int k = tile.k_begin; k < tile.k_end; k += BK, ++it) {
         if (static_cast<int>(it % TRANSFORM_GROUPS) != group) continue;
         const uint32_t stage = it % STAGES2, phase = (it / STAGES2) & 1u;
         // one lane polls the barrier; the warp then proceeds together (the shuffles need all lanes)
@@ -817,29 +887,29 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint32_t local = 0, which = 0;
     bool alive = true;
     const bool use_tma = !(p.accumulate != 0 && sizeof(OutT) == 2);
-    for (int t = cluster_id; t < p.num_tiles && alive; t += num_clusters, ++local) {
-      int m0, n0;
-      decode_tile_pair(p, t, m0, n0);
-      m0 += static_cast<int>(rank) * BM;
+    for (int t = cluster_id; t < num_tiles && alive; t += num_clusters, ++local) {
+      const PairTile tile = decode_pair(p, cum, tiles_m, t);
+      const int m0 = tile.m0 + static_cast<int>(rank) * BM;
+      const int n0 = tile.n0;
       const uint32_t buf = local & 1u;
       const uint32_t use = local >> 1;
       const bool got = mbar_wait(smem_u32(&bars->acc_full[buf]), use & 1u, abort_flag, p.status);
       if (!__all_sync(0xFFFFFFFFu, got)) { alive = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(quarter * 32) << 16);
-      const bool empty_k = p.Kc <= 0;
+      const bool empty_k = tile.k_end <= tile.k_begin;
       auto release = [&]() {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->acc_empty[buf]), 0));
       };
       if (use_tma) {
-        epilogue_tile_tma<OutT>(&tmC, staging_base + static_cast<uint32_t>(warp - 2) * 8192u, which, taddr, m0 + quarter * 32, n0, 0,
-                                static_cast<int>(p.Mo), static_cast<int>(p.No), p.accumulate != 0, empty_k, lane, release);
+        epilogue_tile_tma<OutT>(&tmC, staging_base + static_cast<uint32_t>(warp - 2) * 8192u, which, taddr, m0 + quarter * 32, n0, tile.z,
+                                tile.rows_limit, static_cast<int>(p.No), p.accumulate != 0, empty_k, lane, release);
       } else {
         const int row = m0 + quarter * 32 + lane;
-        const bool row_ok = row < static_cast<int>(p.Mo);
-        OutT* row_ptr = static_cast<OutT*>(p.C) + static_cast<int64_t>(row) * p.ldc;
+        const bool row_ok = row < tile.rows_limit;
+        OutT* row_ptr = static_cast<OutT*>(p.C) + static_cast<int64_t>(tile.z) * p.c_group_stride + static_cast<int64_t>(row) * p.ldc;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t acc[32];
@@ -987,27 +1057,42 @@ cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUten
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   KParams kp{};
   kp.C = a.C;
-  kp.Mo = a.Mo;
+  kp.Mo = a.group_mode == 1 ? a.rows_padded : a.Mo;
   kp.No = a.No;
   kp.Kc = a.Kc;
   kp.ldc = a.ldc;
   kp.c_dtype = a.c_dtype;
   kp.accumulate = a.accumulate ? 1 : 0;
   kp.status = a.status_word;
-  kp.tiles_m = static_cast<int>((a.Mo + 2 * BM - 1) / (2 * BM));
+  kp.group_mode = a.group_mode;
+  kp.G = a.G;
+  kp.offs = a.group_offsets;
+  kp.c_group_stride = a.c_group_stride;
+  const int64_t a_rows_total = kp.Mo;
+  // mode 1: the true number of pair row-tiles is only known on the device (it depends on the segment
+  // lengths); this is an upper bound used for the grid size and the band width
+  kp.tiles_m = static_cast<int>((a_rows_total + 2 * BM - 1) / (2 * BM)) + (a.group_mode == 1 ? a.G : 0);
   kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
-  kp.num_tiles = kp.tiles_m * kp.tiles_n;
-  kp.band = band_rows(2 * BM, a.Kc, kp.tiles_m);
+  kp.num_tiles = kp.tiles_m * kp.tiles_n * (a.group_mode == 2 ? a.G : 1);
+  const int64_t contraction_rows = a.group_mode == 2 ? a.rows_padded : a.Kc;
+  kp.band = band_rows(2 * BM, a.group_mode == 2 ? a.rows_padded / (a.G > 0 ? a.G : 1) : a.Kc, kp.tiles_m);
   CUtensorMap tmA, tmB;
   bool ok;
-  if (a.a_mn_major) ok = make_map(&tmA, a.A, a.Kc, a.Mo, a.lda, 64, BK);
-  else ok = make_map(&tmA, a.A, a.Mo, a.Kc, a.lda, BK, BM);
+  if (a.a_mn_major) ok = make_map(&tmA, a.A, contraction_rows, a.Mo, a.lda, 64, BK);
+  else ok = make_map(&tmA, a.A, a_rows_total, a.Kc, a.lda, BK, BM);
   if (!ok) return cudaErrorInvalidValue;
-  if (a.b_mn_major) ok = make_map(&tmB, a.B, a.Kc, a.No, a.ldb, 64, BK);
-  else ok = make_map(&tmB, a.B, a.No, a.Kc, a.ldb, BK, BN / 2);
+  const int64_t groups_b = a.group_mode == 1 ? a.G : 1;
+  if (a.b_mn_major) {
+    ok = make_map(&tmB, a.B, a.group_mode == 1 ? groups_b * a.Kc : contraction_rows, a.No, a.ldb, 64, BK);
+    kp.b_group_rows = a.Kc;
+  } else {
+    ok = make_map(&tmB, a.B, groups_b * a.No, a.Kc, a.ldb, BK, BN / 2);
+    kp.b_group_rows = a.No;
+  }
   if (!ok) return cudaErrorInvalidValue;
   CUtensorMap tmC;
-  if (!make_map_c(&tmC, a.C, a.c_dtype, 1, a.Mo, a.No, a.ldc, 0)) return cudaErrorInvalidValue;
+  const bool per_group_c = a.group_mode == 2;
+  if (!make_map_c(&tmC, a.C, a.c_dtype, per_group_c ? a.G : 1, kp.Mo, a.No, a.ldc, a.c_group_stride)) return cudaErrorInvalidValue;
   const int clusters = kp.num_tiles < kNumSMs / 2 ? kp.num_tiles : kNumSMs / 2;
   const int grid = 2 * clusters;
   if (a.c_dtype == QF_DT_F32) return launch_pair_majors<float>(a, tmA, tmB, tmC, kp, grid, st);
@@ -1027,9 +1112,19 @@ static int pair_mode() {
 // True if launch_gemm would run this problem on the kernel that can quantize-dequantize staged tiles itself.
 bool gemm_can_fuse(const GemmArgs& a) { return a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode() != 0; }
 
+// Problems the two-CTA kernel takes: plain ones with at least one full 256-row tile, and grouped ones
+// whose expert count fits its shared-memory tile table (segments start on multiples of 128 rows).
+static bool pair_applies(const GemmArgs& a) {
+  if (!pair_mode() || a.Kc <= 0) return false;
+  if (a.group_mode == 0) return a.Mo >= 2 * BM;
+  if (a.G < 1 || a.G > MAX_PAIR_GROUPS) return false;
+  if (a.group_mode == 1) return a.rows_padded >= 2 * BM;
+  return a.Mo >= 2 * BM && a.rows_padded > 0;
+}
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
-  if (a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode()) return launch_gemm_pair(a, st);
+  if (pair_applies(a)) return launch_gemm_pair(a, st);
   if (a.fuse_a_mxfp4 || a.fuse_b_mxfp4) return cudaErrorInvalidValue;       // only the two-CTA kernel fuses (see gemm_can_fuse)
   KParams kp{};
   kp.C = a.C;
