@@ -263,19 +263,14 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-    from paper_2609_39223_b200 import api, synth
+    from paper_2609_39223_b200 import api, replicas, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device — the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
     api.lib()
     peaks = _peaks()
     fmt = api.FMT_MXFP4
@@ -292,8 +287,7 @@ def run_ours(args):
         api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, ws=ws, dX=dX, dW=dW)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     # ---- headline: K steps, inputs resident in HBM -------------------------------------------------
@@ -307,11 +301,7 @@ def run_ours(args):
             step()
         e1.record()
         barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
     status = api.qf_read_status(ws)
     if status != 0:
         raise SystemExit(f"bench.py: device-side status {status} ({api.status_string(status)})")
@@ -415,11 +405,7 @@ def run_ours(args):
         barrier()
         first, last = e2e_run(e2e_steps)
         barrier()
-        e2e_ms = first.elapsed_time(last)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(first.elapsed_time(last), dev)
         e2e = {"value": world * FLOP_PER_STEP * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "how": "pinned host buffers; upload, kernels and download on three streams, two device buffer sets"}
@@ -471,8 +457,7 @@ def run_ours(args):
         if other is not None:
             line["other_workloads"] = other
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish()
 
 
 def main():

@@ -4,4 +4,4 @@ matmul on fake-quantized operands, and the straight-through backward) behind a C
 ``paper_2609_39223_b200.api`` is the thin ctypes binding over ``libqf.so``;
 ``paper_2609_39223_b200.synth`` draws the seeded synthetic workloads.
 """
-__all__ = ["api", "synth"]
+__all__ = ["api", "replicas", "synth"]
