@@ -191,6 +191,12 @@ qf_status_t qf_selftest_cvt(const float* in, int64_t n, uint8_t* e2m1_out, uint8
  * receives the number of differences. */
 qf_status_t qf_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, uint64_t* mismatches, void* stream);
 
+/* Self-test hook for the bounded device-side waits: launches one thread that waits, with the given limit
+ * in SM clock cycles (at most 2^28), on a barrier nothing ever arrives at. The wait gives up, the kernel
+ * returns normally, and the workspace then holds QF_ERR_TIMEOUT in its status word (qf_read_status)
+ * and 1 in its 32-bit word 16. Nothing faults or hangs; the context stays usable. */
+qf_status_t qf_selftest_timeout(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream);
+
 /* Self-test hook for the conversion-free MXFP4 rounding used inside the fused matmul kernel (packed BF16
  * add/subtract of a magic constant): every BF16 bit pattern against every block-scale code in [8, 240]
  * is compared with the conversion-instruction route; *mismatches (device u64) receives the count. */

@@ -25,7 +25,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.qf_fq_linear_fwd_noalloc.restype = c_int
         L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
                                                c_void_p, c_void_p, c_uint32, c_void_p]
+        L.qf_selftest_timeout.restype = c_int
+        L.qf_selftest_timeout.argtypes = [c_void_p, c_size_t, c_int64, c_void_p]
         L.qf_selftest_mxfp4_bf16.restype = c_int
         L.qf_selftest_mxfp4_bf16.argtypes = [c_void_p, c_void_p]
         L.qf_selftest_div.restype = c_int
@@ -280,3 +282,11 @@ def qf_selftest_mxfp4_bf16() -> int:
     out = torch.zeros(1, dtype=torch.int64, device="cuda")
     _check(lib().qf_selftest_mxfp4_bf16(_ptr(out), _stream()), "qf_selftest_mxfp4_bf16")
     return int(out.item())
+
+
+def qf_selftest_timeout(limit_cycles: int = 1 << 20):
+    """Runs the bounded-wait self-test; returns (status word, gave-up flag) read back from the workspace."""
+    ws = workspace(OP_QDQ, 0, 0, 0)
+    _check(lib().qf_selftest_timeout(_ptr(ws), ws.numel(), limit_cycles, _stream()), "qf_selftest_timeout")
+    status = qf_read_status(ws)
+    return status, int(ws.view(torch.int32)[16].item())

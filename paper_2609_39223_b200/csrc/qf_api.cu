@@ -399,6 +399,17 @@ qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_d
                          QF_NOALLOC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
 }
 
+qf_status_t qf_selftest_timeout(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream) {
+  if (!workspace) return QF_ERR_WORKSPACE;
+  if (workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;
+  if (limit_cycles < 1 || limit_cycles > (1ll << 28)) return QF_ERR_SHAPE;      // a fraction of a second at most
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* header = static_cast<uint32_t*>(workspace);
+  if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
+  return cu(launch_selftest_timeout(header + kWsStatus, limit_cycles, reinterpret_cast<int*>(header + 16), st));
+}
+
 qf_status_t qf_selftest_mxfp4_bf16(uint64_t* mismatches, void* stream) {
   if (!mismatches) return QF_ERR_NULL;
   if (qf_status_t s = check_arch()) return s;

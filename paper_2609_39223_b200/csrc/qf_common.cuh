@@ -171,5 +171,6 @@ struct GemmArgs {
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 bool gemm_can_fuse(const GemmArgs& a);
+cudaError_t launch_selftest_timeout(uint32_t* status, long long limit_cycles, int* gave_up, cudaStream_t st);
 
 }  // namespace qf

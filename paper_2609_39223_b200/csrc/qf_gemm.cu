@@ -87,7 +87,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait. Returns false if the CTA is aborting (this wait or another one gave up).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
+                                          long long limit_cycles = kWaitCycles) {
   long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -95,7 +96,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitCycles) break;
+      else if (now - t0 > limit_cycles) break;
     }
   }
   *abort_flag = 1;
@@ -938,6 +939,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing will ever arrive at, with a
+// short limit. The wait must give up, raise the abort flag and record QF_ERR_TIMEOUT; the kernel then
+// returns normally and the context stays usable.
+__global__ void selftest_timeout_kernel(uint32_t* status, long long limit_cycles, int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, limit_cycles);
+    *gave_up = (!ok && abort_flag == 1) ? 1 : 0;
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -1052,6 +1068,11 @@ cudaError_t launch_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUten
 }
 
 }  // namespace
+
+cudaError_t launch_selftest_timeout(uint32_t* status, long long limit_cycles, int* gave_up, cudaStream_t st) {
+  selftest_timeout_kernel<<<1, 32, 0, st>>>(status, limit_cycles, gave_up);
+  return cudaGetLastError();
+}
 
 // Two-CTA path: plain problems whose output has at least one full 256-row pair tile.
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {

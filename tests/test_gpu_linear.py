@@ -246,3 +246,64 @@ def test_in_kernel_mxfp4_quantization_is_bitwise_the_workspace_path(wq, aq, M, N
     assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
     # and against the oracle, like every other path
     _close(y1, oracle.fq_linear_fwd(torch_to_bits(c.X), torch_to_bits(c.W), wq, aq), "Y fused")
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
+    status word and leave the context usable (no trap, no hang)."""
+    status, gave_up = api.qf_selftest_timeout(1 << 20)
+    assert status == 7 and gave_up == 1
+    assert "wait expired" in api.status_string(status)
+    # the context still works
+    x = synth.randn_bf16((4, 64), 1.0, 0, device="cuda")
+    assert torch.equal(api.qf_qdq(api.FMT_MXFP4, x)["out"], api.qf_qdq(api.FMT_MXFP4, x)["out"])
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 8, 32), (257, 136, 96), (511, 264, 160), (127, 8, 32), (1, 16, 64), (640, 72, 4128)])
+def test_edge_shapes_short_and_ragged_contractions(M, N, K):
+    c = synth.linear_case(M, N, K, seed=K, outlier_channels=0)
+    xb, wb, dyb = (torch_to_bits(t) for t in (c.X, c.W, c.dY))
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    fmt = api.FMT_MXFP4
+    _close(api.qf_fq_linear_fwd(X, W, fmt, fmt, y_dtype=torch.float32), oracle.fq_linear_fwd(xb, wb, fmt, fmt), "Y")
+    dx, dw = api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, fmt, fmt)
+    _close(dx, dx_ref, "dX")
+    _close(dw, dw_ref, "dW")
+
+
+def test_bf16_gradient_accumulation_rounds_once():
+    c = synth.linear_case(512, 256, 256, seed=9)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    _, dw32 = api.qf_fq_linear_bwd(dY, X, W, api.FMT_MXFP4, api.FMT_MXFP4, want_dx=False, dw_dtype=torch.float32)
+    base = synth.randn_bf16((256, 256), 1e-2, 10, device="cuda")
+    acc = base.clone()
+    api.qf_fq_linear_bwd(dY, X, W, api.FMT_MXFP4, api.FMT_MXFP4, want_dx=False, dW=acc, flags=api.ACCUMULATE_DW)
+    assert torch.equal(acc, (base.float() + dw32).to(torch.bfloat16))      # one rounding of the FP32 sum
+
+
+def test_grouped_with_more_experts_than_the_pair_kernel_table_holds():
+    E, H, F = 300, 256, 256                   # > 256 experts: served by the one-CTA kernel
+    counts = torch.tensor([(i * 37) % 3 for i in range(E)])              # 0, 1 or 2 blocks of 128 rows
+    offs = torch.zeros(E + 1, dtype=torch.int32); offs[1:] = torch.cumsum(counts * 128, 0)
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 1); W = synth.randn_bf16((E, F, H), 0.02, 2); dYp = synth.randn_bf16((rows, F), 1e-3, 3)
+    y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, api.FMT_MXFP4, api.FMT_MXFP4, dYp)
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_MXFP4, api.FMT_MXFP4, y_dtype=torch.float32)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_MXFP4, api.FMT_MXFP4,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32)
+    _close(y, y_ref, "Y"); _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
+
+
+def test_grouped_odd_block_counts_on_the_pair_kernel():
+    E, H, F = 7, 512, 264                     # segments of 1, 3, 0, 2, 5, 1, 4 blocks: odd ones end in half-used pair tiles
+    counts = torch.tensor([1, 3, 0, 2, 5, 1, 4])
+    offs = torch.zeros(E + 1, dtype=torch.int32); offs[1:] = torch.cumsum(counts * 128, 0)
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 4); W = synth.randn_bf16((E, F, H), 0.02, 5); dYp = synth.randn_bf16((rows, F), 1e-3, 6)
+    y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, api.FMT_MXFP4, api.FMT_MXFP4, dYp)
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_MXFP4, api.FMT_MXFP4, y_dtype=torch.float32)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_MXFP4, api.FMT_MXFP4,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32)
+    _close(y, y_ref, "Y"); _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
+    assert torch.count_nonzero(dw[2]) == 0
