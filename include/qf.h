@@ -151,6 +151,24 @@ qf_status_t qf_fq_grouped_linear_bwd(const void* dY, const void* X, const void* 
                                      float* a_tscale, uint32_t flags, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
+/* Engine-native packing of quantized weights (Section 3.4 "Low-precision weight synchronization",
+ * Section 3.5 "Packing the checkpoint"): a lossless re-layout of what qf_qdq emitted.
+ *   QF_LAYOUT_GGUF_Q4_K (fmt = QF_FMT_Q4_K): `packed` receives rows*cols/256 llama.cpp block_q4_K records
+ *     of 144 bytes {fp16 d, fp16 dmin, 12 bytes of 6-bit scales/offsets, 128 bytes of codes}, row-major.
+ *   QF_LAYOUT_FP4_SWIZZLED_SCALES (fmt = NVFP4 or MXFP4): `packed` receives the block scales in the tiled
+ *     layout block-scaled FP4 tensor-core GEMMs read: scales padded with zeros to multiples of 128 rows and
+ *     4 scale columns, stored tile by tile (tiles row-major, 512 bytes each), byte (r, c) of a tile at
+ *     (r mod 32)*16 + (r div 32)*4 + c. `codes` is ignored: the 4-bit codes are already in the engines'
+ *     layout (two per byte, even element in the low nibble, row-major).
+ * qf_pack_bytes gives the size of `packed`. qf_unpack is the inverse (for Q4_K it fills both codes and
+ * scales; for the FP4 layout only scales). All pointers device, 16-byte aligned. */
+typedef enum { QF_LAYOUT_GGUF_Q4_K = 1, QF_LAYOUT_FP4_SWIZZLED_SCALES = 2 } qf_layout_t;
+size_t qf_pack_bytes(qf_layout_t layout, qf_format_t fmt, int64_t rows, int64_t cols);
+qf_status_t qf_pack(qf_layout_t layout, qf_format_t fmt, const void* codes, const void* scales, int64_t rows, int64_t cols,
+                    void* packed, void* stream);
+qf_status_t qf_unpack(qf_layout_t layout, qf_format_t fmt, const void* packed, int64_t rows, int64_t cols, void* codes,
+                      void* scales, void* stream);
+
 /* Allocation-free forward of the quantization-aware linear layer. (The paper has no counterpart:
  * this is a packaging variant of qf_fq_linear_fwd for hosts that cannot hand the library a workspace.)
  *

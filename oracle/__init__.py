@@ -225,3 +225,33 @@ def fq_linear_bwd(dy, x, w, wq_fmt: int, aq_fmt: int, w_tscale=None, a_tscale=No
     dx = matmul_dgrad(dy, qdq_out(wq_fmt, w, w_tscale))
     dw = matmul_wgrad(dy, qdq_out(aq_fmt, x, a_tscale), n_idx)
     return dx, dw
+
+
+# ---- engine-native packing (the export / weight-synchronisation step) -------------------------------
+
+def pack_gguf_q4k(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    """144-byte llama.cpp Q4_K records from the quantizer's outputs: for each super-block the 16
+    metadata bytes {fp16 d, fp16 dmin, 12 packed 6-bit bytes} followed by its 128 code bytes.
+    codes [rows, cols/2] uint8, scales [rows, cols/256, 16] uint8 -> [rows, cols/256, 144] uint8."""
+    rows, nsb, _ = scales.shape
+    rec = np.empty((rows, nsb, 144), np.uint8)
+    for r in range(rows):
+        for s in range(nsb):
+            rec[r, s, :16] = scales[r, s]
+            rec[r, s, 16:] = codes[r, s * 128:(s + 1) * 128]
+    return rec
+
+
+def swizzle_block_scales(scales: np.ndarray) -> np.ndarray:
+    """FP4 block scales [rows, nblk] in the tiled layout block-scaled tensor-core GEMMs read: padded
+    with zeros to multiples of 128 rows and 4 scale columns; tiles stored row-major, 512 bytes each;
+    inside a tile, byte (r, c) sits at (r mod 32)*16 + (r div 32)*4 + c. Written element by element."""
+    rows, nblk = scales.shape
+    row_tiles, col_tiles = -(-rows // 128), -(-nblk // 4)
+    out = np.zeros(row_tiles * col_tiles * 512, np.uint8)
+    for r in range(rows):
+        for c in range(nblk):
+            tile = (r // 128) * col_tiles + c // 4
+            ri = r % 128
+            out[tile * 512 + (ri % 32) * 16 + (ri // 32) * 4 + c % 4] = scales[r, c]
+    return out

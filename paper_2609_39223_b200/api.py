@@ -25,9 +25,10 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
+LAYOUT_GGUF_Q4_K, LAYOUT_FP4_SWIZZLED_SCALES = 1, 2
 
 
 class QfError(RuntimeError):
@@ -79,6 +80,12 @@ def lib() -> ctypes.CDLL:
         L.qf_fq_linear_fwd_noalloc.restype = c_int
         L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
                                                c_void_p, c_void_p, c_uint32, c_void_p]
+        L.qf_pack_bytes.restype = c_size_t
+        L.qf_pack_bytes.argtypes = [c_int, c_int, c_int64, c_int64]
+        L.qf_pack.restype = c_int
+        L.qf_pack.argtypes = [c_int, c_int, c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
+        L.qf_unpack.restype = c_int
+        L.qf_unpack.argtypes = [c_int, c_int, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
         L.qf_selftest_timeout.restype = c_int
         L.qf_selftest_timeout.argtypes = [c_void_p, c_size_t, c_int64, c_void_p]
         L.qf_selftest_mxfp4_bf16.restype = c_int
@@ -290,3 +297,21 @@ def qf_selftest_timeout(limit_cycles: int = 1 << 20):
     _check(lib().qf_selftest_timeout(_ptr(ws), ws.numel(), limit_cycles, _stream()), "qf_selftest_timeout")
     status = qf_read_status(ws)
     return status, int(ws.view(torch.int32)[16].item())
+
+
+def qf_pack_bytes(layout: int, fmt: int, rows: int, cols: int) -> int:
+    return int(lib().qf_pack_bytes(layout, fmt, rows, cols))
+
+
+def qf_pack(layout: int, fmt: int, codes, scales, rows: int, cols: int) -> torch.Tensor:
+    """Engine-native re-layout of quantized weights: GGUF Q4_K records, or swizzled FP4 block scales."""
+    packed = torch.empty(qf_pack_bytes(layout, fmt, rows, cols), dtype=torch.uint8, device=scales.device)
+    _check(lib().qf_pack(layout, fmt, _ptr(codes), _ptr(scales), rows, cols, _ptr(packed), _stream()), "qf_pack")
+    return packed
+
+
+def qf_unpack(layout: int, fmt: int, packed: torch.Tensor, rows: int, cols: int):
+    codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=packed.device) if layout == LAYOUT_GGUF_Q4_K else None
+    scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=packed.device)
+    _check(lib().qf_unpack(layout, fmt, _ptr(packed), rows, cols, _ptr(codes), _ptr(scales), _stream()), "qf_unpack")
+    return codes, scales

@@ -399,6 +399,45 @@ qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_d
                          QF_NOALLOC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
 }
 
+static qf_status_t check_pack(int layout, int fmt, int64_t rows, int64_t cols) {
+  if (layout == QF_LAYOUT_GGUF_Q4_K) { if (fmt != QF_FMT_Q4_K) return QF_ERR_FORMAT; }
+  else if (layout == QF_LAYOUT_FP4_SWIZZLED_SCALES) { if (fmt != QF_FMT_NVFP4 && fmt != QF_FMT_MXFP4) return QF_ERR_FORMAT; }
+  else return QF_ERR_FORMAT;
+  if (rows < 0 || cols < 0 || cols % block_of(fmt)) return QF_ERR_SHAPE;
+  return QF_OK;
+}
+
+size_t qf_pack_bytes(qf_layout_t layout, qf_format_t fmt, int64_t rows, int64_t cols) {
+  if (check_pack(layout, fmt, rows, cols) != QF_OK) return 0;
+  if (layout == QF_LAYOUT_GGUF_Q4_K) return static_cast<size_t>(rows) * (cols / 256) * 144;
+  const int64_t nblk = cols / block_of(fmt);
+  return static_cast<size_t>((rows + 127) / 128) * ((nblk + 3) / 4) * 512;
+}
+
+qf_status_t qf_pack(qf_layout_t layout, qf_format_t fmt, const void* codes, const void* scales, int64_t rows, int64_t cols,
+                    void* packed, void* stream) {
+  if (qf_status_t s = check_pack(layout, fmt, rows, cols)) return s;
+  const bool empty = rows == 0 || cols == 0;
+  if (!empty && (!scales || !packed || (layout == QF_LAYOUT_GGUF_Q4_K && !codes))) return QF_ERR_NULL;
+  if (!aligned16(scales) || !aligned16(packed) || (layout == QF_LAYOUT_GGUF_Q4_K && !aligned16(codes))) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (layout == QF_LAYOUT_GGUF_Q4_K) return cu(launch_pack_q4k(codes, scales, rows * (cols / 256), packed, false, nullptr, nullptr, st));
+  return cu(launch_swizzle_scales(scales, rows, cols / block_of(fmt), packed, false, st));
+}
+
+qf_status_t qf_unpack(qf_layout_t layout, qf_format_t fmt, const void* packed, int64_t rows, int64_t cols, void* codes,
+                      void* scales, void* stream) {
+  if (qf_status_t s = check_pack(layout, fmt, rows, cols)) return s;
+  const bool empty = rows == 0 || cols == 0;
+  if (!empty && (!scales || !packed || (layout == QF_LAYOUT_GGUF_Q4_K && !codes))) return QF_ERR_NULL;
+  if (!aligned16(scales) || !aligned16(packed) || (layout == QF_LAYOUT_GGUF_Q4_K && !aligned16(codes))) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (layout == QF_LAYOUT_GGUF_Q4_K) return cu(launch_pack_q4k(nullptr, nullptr, rows * (cols / 256), const_cast<void*>(packed), true, codes, scales, st));
+  return cu(launch_swizzle_scales(packed, rows, cols / block_of(fmt), scales, true, st));
+}
+
 qf_status_t qf_selftest_timeout(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream) {
   if (!workspace) return QF_ERR_WORKSPACE;
   if (workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;

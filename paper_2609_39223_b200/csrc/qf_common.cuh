@@ -169,6 +169,9 @@ struct GemmArgs {
   bool fuse_a_mxfp4, fuse_b_mxfp4;   // apply the MXFP4 quantize-dequantize to the staged tiles inside the kernel
 };
 
+cudaError_t launch_pack_q4k(const void* codes, const void* scales, int64_t nsb, void* records, bool unpack, void* codes_out,
+                            void* scales_out, cudaStream_t st);
+cudaError_t launch_swizzle_scales(const void* scales, int64_t rows, int64_t nblk, void* out, bool unswizzle, cudaStream_t st);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 bool gemm_can_fuse(const GemmArgs& a);
 cudaError_t launch_selftest_timeout(uint32_t* status, long long limit_cycles, int* gave_up, cudaStream_t st);
