@@ -122,7 +122,8 @@ def _oracle_slice(m_rows: int, n_rows: int, seed: int = 0):
     import oracle
     from paper_2609_39223_b200 import synth
     c = synth.linear_case(m_rows, n_rows, K, seed=seed)
-    to_bits = lambda t: t.contiguous().view(__import__("torch").int16).numpy().view(np.uint16)
+    import torch
+    to_bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
     xb, wb, dyb = to_bits(c.X), to_bits(c.W), to_bits(c.dY)
     t0 = time.perf_counter()
     oracle.fq_linear_fwd(xb, wb, oracle.FMT_MXFP4, oracle.FMT_MXFP4)
@@ -445,7 +446,7 @@ def run_ours(args):
             "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel (tcgen05 cta_group::2 BF16, 256x256x64 tiles per CTA pair)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
                          # mean dram__bytes_read.sum + dram__bytes_write.sum per launch over the three matmuls of a
-                         # step, from the full-size ncu capture summarised in profiles/gemm_pair_kernel_mxfp4_linear.md
+                         # step, from an ncu capture of this workload (summary committed with the other profiles)
                          "traffic": 916.2e6 if (M, N, K) == (8192, 12288, 4096) else None,
                          "peak_source": f"{peaks['source']} cuBLAS bf16 burst", "ms_per_launch": gemm_ms,
                          "frac_of_sustained": achieved / peaks["bf16_sustained"] if achieved else None,

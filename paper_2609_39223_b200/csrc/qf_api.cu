@@ -79,9 +79,12 @@ qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t col
   return cu(launch_qdq(q, st));
 }
 
-qf_status_t check_linear_common(const void* W, int64_t M, int64_t N, int64_t K, int wq, int aq, const float* w_ts,
+// Checks shared by the forward and backward calls. W may be NULL only when the caller does not need it
+// (a backward call that asks for dW alone): need_w says whether it is required.
+qf_status_t check_linear_common(const void* W, bool need_w, int64_t M, int64_t N, int64_t K, int wq, int aq, const float* w_ts,
                                 const float* a_ts, uint32_t flags, void* ws, size_t ws_bytes, int64_t groups) {
-  if (!W || !ws) return !W ? QF_ERR_NULL : QF_ERR_WORKSPACE;
+  if (need_w && !W) return QF_ERR_NULL;
+  if (!ws) return QF_ERR_WORKSPACE;
   if (M < 0 || N < 0 || K < 0) return QF_ERR_SHAPE;
   if (!valid_fmt(wq, true) || !valid_fmt(aq, true)) return QF_ERR_FORMAT;
   if (aq == QF_FMT_Q4_K) return QF_ERR_FORMAT;                    // Q4_K is a weight-only format
@@ -90,7 +93,7 @@ qf_status_t check_linear_common(const void* W, int64_t M, int64_t N, int64_t K, 
   if (aq != QF_FMT_NONE && K % block_of(aq)) return QF_ERR_SHAPE;
   if (wq == QF_FMT_NVFP4 && (flags & QF_W_TSCALE_GIVEN) && !w_ts) return QF_ERR_NULL;
   if (aq == QF_FMT_NVFP4 && (flags & QF_A_TSCALE_GIVEN) && !a_ts) return QF_ERR_NULL;
-  if (!aligned16(W) || !aligned16(ws)) return QF_ERR_ALIGN;
+  if ((W && !aligned16(W)) || !aligned16(ws)) return QF_ERR_ALIGN;
   if (ws_bytes < linear_ws_bytes(M, N, K, groups)) return QF_ERR_WORKSPACE;
   return QF_OK;
 }
@@ -105,7 +108,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   const int64_t groups = grouped ? G : 1;
   if (!X || !Y) return QF_ERR_NULL;
   if (!valid_dtype(y_dtype)) return QF_ERR_DTYPE;
-  if (qf_status_t s = check_linear_common(W, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
+  if (qf_status_t s = check_linear_common(W, true, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
   if (!aligned16(X) || !aligned16(Y)) return QF_ERR_ALIGN;
   if (qf_status_t s = check_arch()) return s;
   if (M == 0 || N == 0) return QF_OK;
@@ -153,8 +156,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
   if (!dX && !dW) return QF_ERR_NULL;
   if (dW && !X) return QF_ERR_NULL;
   if ((dX && !valid_dtype(dx_dtype)) || (dW && !valid_dtype(dw_dtype))) return QF_ERR_DTYPE;
-  if (qf_status_t s = check_linear_common(W ? W : dY, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
-  if (dX && !W) return QF_ERR_NULL;
+  if (qf_status_t s = check_linear_common(W, dX != nullptr, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
   if (!aligned16(dY) || (X && !aligned16(X)) || (dX && !aligned16(dX)) || (dW && !aligned16(dW))) return QF_ERR_ALIGN;
   if (qf_status_t s = check_arch()) return s;
   if (M == 0 || N == 0 || K == 0) {

@@ -34,14 +34,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-__device__ __forceinline__ uint32_t habs2_bits(uint32_t w) { return w & 0x7FFF7FFFu; }
-
-// max of two packed pairs of non-negative BF16 values (bit patterns of non-negative floats are
-// ordered like unsigned integers)
-__device__ __forceinline__ uint32_t umax2_bits(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
-
-__device__ __forceinline__ uint32_t hmax_of_pair(uint32_t w) { return max(w & 0xFFFFu, w >> 16); }
-
 // E2M1 pair: lo -> low nibble, hi -> high nibble; round to nearest even, saturate to +-6.
 __device__ __forceinline__ uint32_t e2m1x2_encode(float lo, float hi) {
   return static_cast<uint32_t>(__nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest)) & 0xFFu;

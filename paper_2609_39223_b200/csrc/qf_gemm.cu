@@ -17,7 +17,6 @@
 // teardown (the producer first gives its outstanding copies a bounded chance to land), tensor
 // memory is released and the kernel returns.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "qf_common.cuh"
 
@@ -1120,23 +1119,13 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   return launch_pair_majors<__nv_bfloat16>(a, tmA, tmB, tmC, kp, grid, st);
 }
 
-static int pair_mode() {
-  // QF_GEMM_PAIR=0 forces the one-CTA kernel (A/B comparison in profiling runs); default: two-CTA when it applies
-  static int mode = -1;
-  if (mode < 0) {
-    const char* e = getenv("QF_GEMM_PAIR");
-    mode = (e && e[0] == '0') ? 0 : 1;
-  }
-  return mode;
-}
-
 // True if launch_gemm would run this problem on the kernel that can quantize-dequantize staged tiles itself.
-bool gemm_can_fuse(const GemmArgs& a) { return a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0 && pair_mode() != 0; }
+bool gemm_can_fuse(const GemmArgs& a) { return a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0; }
 
 // Problems the two-CTA kernel takes: plain ones with at least one full 256-row tile, and grouped ones
 // whose expert count fits its shared-memory tile table (segments start on multiples of 128 rows).
 static bool pair_applies(const GemmArgs& a) {
-  if (!pair_mode() || a.Kc <= 0) return false;
+  if (a.Kc <= 0) return false;
   if (a.group_mode == 0) return a.Mo >= 2 * BM;
   if (a.G < 1 || a.G > MAX_PAIR_GROUPS) return false;
   if (a.group_mode == 1) return a.rows_padded >= 2 * BM;

@@ -17,11 +17,7 @@ constexpr int kThreads = 256;
 __device__ __forceinline__ uint4 ld_chunk(const uint4* p) { return __ldg(p); }
 
 // max |x| over the 8 BF16 values of a chunk, as BF16 bits (sign clear)
-__device__ __forceinline__ uint32_t chunk_amax_bits(const uint4& v) {
-  uint32_t m = umax2_bits(umax2_bits(habs2_bits(v.x), habs2_bits(v.y)),
-                          umax2_bits(habs2_bits(v.z), habs2_bits(v.w)));
-  return hmax_of_pair(m);
-}
+__device__ __forceinline__ uint32_t chunk_amax_bits(const uint4& v) { return chunk8_amax_bits(v.x, v.y, v.z, v.w); }
 
 // ---------------------------------------------------------------------------------------------
 // tensor amax
