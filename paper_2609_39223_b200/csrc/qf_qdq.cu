@@ -259,6 +259,9 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restri
 // x_hat = (d * s6) * C - (dmin * m6)  (Eq. q4k-dequant); min/max affine rule for the quantizer.
 // ---------------------------------------------------------------------------------------------
 
+#ifndef QF_Q4K_MINBLOCKS
+#define QF_Q4K_MINBLOCKS 5      // 48 registers: five resident blocks per SM measured 4% faster than four
+#endif
 constexpr float kRcp15 = 1.0f / 15.0f;        // correctly rounded reciprocals of the two constant divisors
 constexpr float kRcp63 = 1.0f / 63.0f;
 constexpr float kRound = 12582912.0f;      // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
@@ -316,7 +319,7 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
   }
 }
 
-__global__ void __launch_bounds__(kThreads) qdq_q4k_kernel(const uint4* __restrict__ in, int64_t nsub,
+__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(const uint4* __restrict__ in, int64_t nsub,
                                                            uint4* __restrict__ out, uint4* __restrict__ codes,
                                                            uint4* __restrict__ scales) {
   const int lane = threadIdx.x & 31;
