@@ -136,7 +136,10 @@ qf_status_t qf_fq_linear_bwd(const void* dY, const void* X, const void* W, void*
  * the same quantization-aware layer). Rows of X are sorted by expert; group_offsets is a device
  * int32[G+1] of segment starts, each a multiple of 128 (the caller pads segments with zero rows;
  * a zero row quantizes to a zero row in every format); rows_padded = group_offsets[G].
- * W is [G,N,K], Y is [rows_padded,N]:  Y[r,:] = X_hat[r,:] . W_hat[g(r)]^T. */
+ * W is [G,N,K], Y is [rows_padded,N]:  Y[r,:] = X_hat[r,:] . W_hat[g(r)]^T.
+ * NVFP4 weights: every expert is its own tensor with its own tensor scale, so w_tscale is an array of G
+ * floats (required; read if QF_W_TSCALE_GIVEN, otherwise written). An NVFP4 activation scale is a
+ * single float for the whole of X (the experts share one input-activation scale). */
 qf_status_t qf_fq_grouped_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype,
                                      const int32_t* group_offsets, int G, int64_t rows_padded, int64_t N,
                                      int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,

@@ -60,14 +60,19 @@ Workspace carve(void* ws, int64_t N, int64_t K, int64_t groups) {
 }
 
 // Fake-quantize one operand into `dst` (BF16, same shape). NVFP4 derives or reads its tensor scale.
+// `groups` > 1 (NVFP4 weights of a grouped layer): every expert has its own tensor scale, tscale_user is an
+// array of `groups` floats (required).
 qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t cols, void* dst, float* tscale_user,
-                             bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st) {
+                             bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st,
+                             int groups = 1) {
   QdqArgs q{};
   q.fmt = fmt;
   q.in = src;
   q.rows = rows;
   q.cols = cols;
   q.out = dst;
+  q.groups = fmt == QF_FMT_NVFP4 ? groups : 1;
+  if (fmt == QF_FMT_NVFP4 && groups > 1 && !tscale_user) return QF_ERR_NULL;
   if (fmt == QF_FMT_NVFP4) {
     if (tscale_given) {
       q.tscale_in = tscale_user;
@@ -131,7 +136,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   const void* Xh = X;
   if (K > 0) {
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
       Wh = w.w_hat;
     }
     if (a_amax_out) {
@@ -182,7 +187,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && wq == QF_FMT_MXFP4 && gemm_can_fuse(g);
     const void* Wh = W;
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st)) return s;
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
       Wh = w.w_hat;
     }
     g.B = Wh;

@@ -124,6 +124,7 @@ struct QdqArgs {
   const uint32_t* amax_bits;     // NVFP4: tensor amax as FP32 bits (device) to derive it from
   float* tscale_out;             // NVFP4: where the derived scale is written (nullable)
   bool reverse;                  // walk the tensor back to front (after an amax pass: L2 holds the tail)
+  int groups;                    // NVFP4: > 1 = that many equal tensors back to back, each with its own tensor scale
 };
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);

@@ -26,6 +26,9 @@ __device__ __forceinline__ uint32_t chunk_amax_bits(const uint4& v) { return chu
 __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t nchunks,
                                                         const __nv_bfloat16* __restrict__ tail, int ntail,
                                                         uint32_t* __restrict__ amax_bits) {
+  // gridDim.y > 1: one tensor per y-slice (the experts of a grouped layer), nchunks chunks each
+  in += static_cast<int64_t>(blockIdx.y) * nchunks;
+  amax_bits += blockIdx.y;
   uint32_t m = 0;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
   int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
@@ -188,15 +191,23 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restri
                                                            const float* __restrict__ tscale_in,
                                                            const uint32_t* __restrict__ amax_bits,
                                                            float* __restrict__ tscale_out, int reverse) {
+  // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
+  {
+    const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
+    in += 2 * goff;
+    if (out) out += 2 * goff;
+    if (codes) codes += goff;
+    if (scales) scales += FMT == QF_FMT_NVFP4 ? goff : goff / 2;
+  }
   float s_t = 1.0f, denom = 6.0f, rc_denom = 0.0f;
   bool denom_safe = false;
   if (FMT == QF_FMT_NVFP4) {
     if (amax_bits) {
-      const float amax_t = __uint_as_float(*amax_bits);
+      const float amax_t = __uint_as_float(amax_bits[blockIdx.y]);
       s_t = amax_t == 0.0f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);            // 2688 = 6 * 448
-      if (tscale_out && blockIdx.x == 0 && threadIdx.x == 0) *tscale_out = s_t;
+      if (tscale_out && blockIdx.x == 0 && threadIdx.x == 0) tscale_out[blockIdx.y] = s_t;
     } else {
-      s_t = *tscale_in;
+      s_t = tscale_in[blockIdx.y];
     }
     denom = __fmul_rn(6.0f, s_t);
     denom_safe = div_safe(denom);
@@ -537,6 +548,17 @@ int capped_grid(int64_t items, int per_thread, int blocks_per_sm) {
 
 }  // namespace
 
+// G tensors of n elements each, stored back to back (n a multiple of 8): amax_bits[g] = max |x| of tensor g
+cudaError_t launch_amax_grouped(const void* in, int64_t n, int G, uint32_t* amax_bits, cudaStream_t st) {
+  const int64_t nchunks = n / 8;
+  if (G <= 0 || nchunks == 0) return cudaSuccess;
+  int gx = grid_for(nchunks, 4);
+  const int cap = (kNumSMs * 8 + G - 1) / G;
+  if (gx > cap) gx = cap < 1 ? 1 : cap;
+  amax_kernel<<<dim3(gx, G), kThreads, 0, st>>>(static_cast<const uint4*>(in), nchunks, nullptr, 0, amax_bits);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st) {
   const int64_t nchunks = n / 8;
   const int ntail = static_cast<int>(n % 8);
@@ -558,8 +580,11 @@ cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st) {
   const uint4* in = static_cast<const uint4*>(a.in);
   uint4* out = static_cast<uint4*>(a.out);
   if (a.fmt == QF_FMT_NVFP4) {
-    const int64_t nunits = nelem / 16;
-    qdq_fp4_kernel<QF_FMT_NVFP4><<<capped_grid(nunits, kUnitsPerThread, 16), kThreads, 0, st>>>(
+    const int slices = a.groups > 1 ? a.groups : 1;
+    const int64_t nunits = nelem / 16 / slices;
+    int gx = capped_grid(nunits, kUnitsPerThread, 16);
+    if (slices > 1 && gx > (kNumSMs * 16 + slices - 1) / slices) gx = (kNumSMs * 16 + slices - 1) / slices;
+    qdq_fp4_kernel<QF_FMT_NVFP4><<<dim3(gx, slices), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), a.tscale_in, a.amax_bits, a.tscale_out,
         a.reverse ? 1 : 0);
   } else if (a.fmt == QF_FMT_MXFP4) {
@@ -580,11 +605,20 @@ cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st) {
 // barrier was tried for tensors under 10 MB and measured no faster (12.3 us against 12.3 us for
 // 2048 x 2048), because at that size L2 already serves the second read; it was dropped.
 cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st) {
+  QdqArgs q = a;
+  q.tscale_in = nullptr;
+  if (a.groups > 1) {
+    // per-expert tensor scales: the caller's scale array doubles as the amax accumulator (FP32 bits of a
+    // non-negative value), which the quantize pass then overwrites with the derived scales
+    uint32_t* bits = reinterpret_cast<uint32_t*>(a.tscale_out);
+    if (cudaError_t e = cudaMemsetAsync(bits, 0, sizeof(uint32_t) * a.groups, st)) return e;
+    if (cudaError_t e = launch_amax_grouped(a.in, a.rows * a.cols / a.groups, a.groups, bits, st)) return e;
+    q.amax_bits = bits;
+    return launch_qdq(q, st);
+  }
   uint32_t* amax_bits = header + amax_word;
   if (cudaError_t e = launch_amax(a.in, a.rows * a.cols, amax_bits, st)) return e;
-  QdqArgs q = a;
   q.amax_bits = amax_bits;
-  q.tscale_in = nullptr;
   q.reverse = true;
   return launch_qdq(q, st);
 }

@@ -307,3 +307,25 @@ def test_grouped_odd_block_counts_on_the_pair_kernel():
                                           dx_dtype=torch.float32, dw_dtype=torch.float32)
     _close(y, y_ref, "Y"); _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
     assert torch.count_nonzero(dw[2]) == 0
+
+
+def test_grouped_nvfp4_weights_have_one_tensor_scale_per_expert():
+    E, H, F = 5, 256, 264
+    counts = torch.tensor([2, 1, 0, 3, 1])
+    offs = torch.zeros(E + 1, dtype=torch.int32); offs[1:] = torch.cumsum(counts * 128, 0)
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 11)
+    W = synth.randn_bf16((E, F, H), 0.02, 12)
+    W = (W.float() * torch.tensor([1.0, 4.0, 0.25, 16.0, 0.5]).view(E, 1, 1)).to(torch.bfloat16)     # experts of different magnitude
+    dYp = synth.randn_bf16((rows, F), 1e-3, 13)
+    y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, api.FMT_NVFP4, api.FMT_NONE, dYp)
+    wts = torch.zeros(E, device="cuda")
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NONE, y_dtype=torch.float32, w_tscale=wts)
+    want = [np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(W[g]))["tensor_scale"]) for g in range(E)]
+    assert [np.float32(v) for v in wts.cpu().tolist()] == want
+    _close(y, y_ref, "Y")
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NONE,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32, w_tscale=wts, flags=api.W_TSCALE_GIVEN)
+    _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
+    with pytest.raises(api.QfError):          # the per-expert scale array is required
+        api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NONE)
