@@ -64,6 +64,7 @@ typedef enum {
 #define QF_W_TSCALE_GIVEN 0x1u     /* linear calls: *w_tscale is an input (tied / shared scale)      */
 #define QF_A_TSCALE_GIVEN 0x2u     /* linear calls: *a_tscale is an input (running activation scale) */
 #define QF_ACCUMULATE_DW 0x4u      /* backward: dW += ... instead of dW = ... (gradient accumulation) */
+#define QF_AMAX_RUNNING 0x10u      /* qf_nvfp4_tensor_scale: the incoming *amax_state takes part in the maximum        */
 #define QF_FUSED_QDQ 0x8u          /* linear calls: quantize-dequantize MXFP4 operands inside the matmul kernel, on the
                                       tiles staged in shared memory, instead of writing fake-quantized copies to the
                                       workspace first. Same results bit for bit. Applies to MXFP4 operands of
@@ -108,6 +109,19 @@ qf_status_t qf_dequant(qf_format_t fmt, const void* codes, const void* scales, c
 /* Tensor-wide max |x| of a BF16 tensor of n elements, written as FP32 to *amax_out (the statistic
  * the NVFP4 tensor scale and the trainer's running activation maximum are derived from). */
 qf_status_t qf_amax(const void* in, int64_t n, float* amax_out, void* stream);
+
+/* NVFP4 tensor scales that span more than one tensor or more than one step ("Engine-specific scale
+ * sharing"; the NVFP4 paragraph on the running activation maximum): fused projections (query/key/value,
+ * gate/up) share one weight tensor scale computed over their concatenation and one activation scale, and
+ * the activation scale exported with the checkpoint is derived from a running absolute maximum.
+ *   tensors / sizes  HOST arrays of n device pointers to BF16 tensors and their element counts.
+ *   amax_state       device float*, in/out: receives max |x| over all listed tensors; with QF_AMAX_RUNNING
+ *                    its previous value takes part in the maximum (running maximum across calls; it must
+ *                    then hold a non-negative finite value, e.g. 0 before the first step).
+ *   scale_out        device float*, nullable: receives amax_state/(6*448), or 1.0 when the maximum is 0 -
+ *                    the value to hand to qf_qdq / the linear calls as a given tensor scale. */
+qf_status_t qf_nvfp4_tensor_scale(const void* const* tensors, const int64_t* sizes, int n, float* amax_state, float* scale_out,
+                                  uint32_t flags, void* stream);
 
 /* Quantization-aware linear layer, forward (Eq. fakequant):
  *     Y[M,N] = Q_a^-1(Q_a(X[M,K])) . Q_w^-1(Q_w(W[N,K]))^T,   BF16 operands, FP32 accumulation.

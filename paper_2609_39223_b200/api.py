@@ -16,7 +16,7 @@ FMT_NONE, FMT_NVFP4, FMT_MXFP4, FMT_Q4_K = 0, 1, 2, 3
 DT_BF16, DT_F32 = 0, 1
 OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 3, 4
 TENSOR_SCALE_GIVEN = 0x1
-W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ = 0x1, 0x2, 0x4, 0x8
+W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x2, 0x4, 0x8, 0x10
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 
@@ -25,7 +25,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack", "qf_nvfp4_tensor_scale",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 LAYOUT_GGUF_Q4_K, LAYOUT_FP4_SWIZZLED_SCALES = 1, 2
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.qf_fq_linear_fwd_noalloc.restype = c_int
         L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
                                                c_void_p, c_void_p, c_uint32, c_void_p]
+        L.qf_nvfp4_tensor_scale.restype = c_int
+        L.qf_nvfp4_tensor_scale.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint32, c_void_p]
         L.qf_pack_bytes.restype = c_size_t
         L.qf_pack_bytes.argtypes = [c_int, c_int, c_int64, c_int64]
         L.qf_pack.restype = c_int
@@ -315,3 +317,15 @@ def qf_unpack(layout: int, fmt: int, packed: torch.Tensor, rows: int, cols: int)
     scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=packed.device)
     _check(lib().qf_unpack(layout, fmt, _ptr(packed), rows, cols, _ptr(codes), _ptr(scales), _stream()), "qf_unpack")
     return codes, scales
+
+
+def qf_nvfp4_tensor_scale(tensors, amax_state: torch.Tensor, *, running: bool = False, want_scale: bool = True):
+    """Shared NVFP4 tensor scale over several BF16 tensors (fused projections) and/or over steps (running
+    activation maximum). Updates ``amax_state`` (1-element float32 CUDA tensor) and returns the scale tensor."""
+    n = len(tensors)
+    ptrs = (c_void_p * max(n, 1))(*[t.data_ptr() for t in tensors])
+    sizes = (c_int64 * max(n, 1))(*[t.numel() for t in tensors])
+    scale = torch.empty(1, dtype=torch.float32, device=amax_state.device) if want_scale else None
+    _check(lib().qf_nvfp4_tensor_scale(ptrs, sizes, n, _ptr(amax_state), _ptr(scale), AMAX_RUNNING if running else 0, _stream()),
+           "qf_nvfp4_tensor_scale")
+    return scale

@@ -323,6 +323,27 @@ qf_status_t qf_amax(const void* in, int64_t n, float* amax_out, void* stream) {
   return cu(launch_amax(in, n, reinterpret_cast<uint32_t*>(amax_out), st));
 }
 
+qf_status_t qf_nvfp4_tensor_scale(const void* const* tensors, const int64_t* sizes, int n, float* amax_state, float* scale_out,
+                                  uint32_t flags, void* stream) {
+  if (n < 0) return QF_ERR_SHAPE;
+  if (!amax_state || (n > 0 && (!tensors || !sizes))) return QF_ERR_NULL;
+  for (int i = 0; i < n; ++i) {
+    if (sizes[i] < 0) return QF_ERR_SHAPE;
+    if (sizes[i] > 0 && !tensors[i]) return QF_ERR_NULL;
+    if (!aligned16(tensors[i])) return QF_ERR_ALIGN;
+  }
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the state word is the accumulator: FP32 bits of a non-negative value order like unsigned integers
+  if (!(flags & QF_AMAX_RUNNING))
+    if (cudaError_t e = cudaMemsetAsync(amax_state, 0, 4, st)) return cu(e);
+  for (int i = 0; i < n; ++i)
+    if (sizes[i] > 0)
+      if (cudaError_t e = launch_amax(tensors[i], sizes[i], reinterpret_cast<uint32_t*>(amax_state), st)) return cu(e);
+  if (scale_out) return cu(launch_amax_to_scale(reinterpret_cast<const uint32_t*>(amax_state), scale_out, st));
+  return QF_OK;
+}
+
 qf_status_t qf_fq_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N, int64_t K,
                              qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale, float* a_amax_out,
                              uint32_t flags, void* workspace, size_t workspace_bytes, void* stream) {

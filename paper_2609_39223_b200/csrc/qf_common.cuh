@@ -129,6 +129,7 @@ struct QdqArgs {
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);
 cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStream_t st);
+cudaError_t launch_amax_to_scale(const uint32_t* amax_bits, float* scale, cudaStream_t st);
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st);
 cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st);
 cudaError_t launch_dequant(int fmt, const void* codes, const void* scales, const float* tscale, int64_t rows,

@@ -53,6 +53,12 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
 
 __global__ void amax_to_float_kernel(const uint32_t* amax_bits, float* out) { *out = __uint_as_float(*amax_bits); }
 
+// s = amax / (6 * 448), 1.0 for an all-zero tensor: the NVFP4 tensor scale that goes with an absolute maximum
+__global__ void amax_to_scale_kernel(const uint32_t* amax_bits, float* scale) {
+  const float a = __uint_as_float(*amax_bits);
+  *scale = a == 0.0f ? 1.0f : __fdiv_rn(a, 2688.0f);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Exact division without the per-element IEEE divide sequence.
 //
@@ -565,6 +571,11 @@ cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStre
   amax_kernel<<<grid_for(nchunks, 4), kThreads, 0, st>>>(static_cast<const uint4*>(in), nchunks,
                                                          static_cast<const __nv_bfloat16*>(in) + nchunks * 8, ntail,
                                                          amax_bits);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_amax_to_scale(const uint32_t* amax_bits, float* scale, cudaStream_t st) {
+  amax_to_scale_kernel<<<1, 1, 0, st>>>(amax_bits, scale);
   return cudaGetLastError();
 }
 

@@ -205,3 +205,26 @@ def test_large_ragged_tensor_stays_inside_its_buffers(fmt, name):
 
 def test_conversion_free_mxfp4_rounding_matches_the_conversion_route_exhaustively():
     assert api.qf_selftest_mxfp4_bf16() == 0
+
+
+def test_tied_tensor_scale_over_fused_projections_and_running_activation_maximum():
+    # one weight scale for q/k/v computed over their concatenation: each quantizes as a slice of the concatenation would
+    q = synth.randn_bf16((64, 256), 0.02, 1); k = synth.randn_bf16((16, 256), 0.05, 2); v = synth.randn_bf16((16, 256), 0.01, 3)
+    state = torch.zeros(1, device="cuda")
+    scale = api.qf_nvfp4_tensor_scale([q.cuda(), k.cuda(), v.cuda()], state)
+    cat = torch.cat([q, k, v])
+    whole = oracle.qdq(api.FMT_NVFP4, torch_to_bits(cat))
+    assert np.float32(scale.item()) == whole["tensor_scale"] and state.item() == cat.abs().max().item()
+    parts = [api.qf_qdq(api.FMT_NVFP4, t.cuda(), tensor_scale=scale) for t in (q, k, v)]
+    np.testing.assert_array_equal(np.concatenate([torch_to_bits(p["out"]) for p in parts]), whole["out"])
+    np.testing.assert_array_equal(np.concatenate([p["codes"].cpu().numpy() for p in parts]), whole["codes"])
+    # running maximum of an activation across steps
+    state.zero_()
+    seen = 0.0
+    for step, std in enumerate((1.0, 3.0, 0.5)):
+        x = synth.randn_bf16((128, 256), std, 10 + step, device="cuda")
+        s = api.qf_nvfp4_tensor_scale([x], state, running=True)
+        seen = max(seen, x.abs().max().item())
+        assert state.item() == seen and np.float32(s.item()) == np.float32(seen) / np.float32(2688.0)
+    zero = api.qf_nvfp4_tensor_scale([torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")], torch.zeros(1, device="cuda"))
+    assert zero.item() == 1.0
