@@ -64,6 +64,10 @@ typedef enum {
 #define QF_W_TSCALE_GIVEN 0x1u     /* linear calls: *w_tscale is an input (tied / shared scale)      */
 #define QF_A_TSCALE_GIVEN 0x2u     /* linear calls: *a_tscale is an input (running activation scale) */
 #define QF_ACCUMULATE_DW 0x4u      /* backward: dW += ... instead of dW = ... (gradient accumulation) */
+#define QF_REUSE_W_HAT 0x20u       /* linear calls: the workspace still holds the fake-quantized W written by an earlier call */
+#define QF_REUSE_X_HAT 0x40u       /* with the same tensor, formats and shapes (e.g. the forward of this step): skip its
+                                      recomputation. The paper's layer discards these copies after the forward matmul and
+                                      recomputes them; keeping the workspace alive trades that memory for two passes. */
 #define QF_AMAX_RUNNING 0x10u      /* qf_nvfp4_tensor_scale: the incoming *amax_state takes part in the maximum        */
 #define QF_FUSED_QDQ 0x8u          /* linear calls: quantize-dequantize MXFP4 operands inside the matmul kernel, on the
                                       tiles staged in shared memory, instead of writing fake-quantized copies to the

@@ -17,6 +17,7 @@ DT_BF16, DT_F32 = 0, 1
 OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 3, 4
 TENSOR_SCALE_GIVEN = 0x1
 W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x2, 0x4, 0x8, 0x10
+REUSE_W_HAT, REUSE_X_HAT = 0x20, 0x40
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 

@@ -136,7 +136,8 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   const void* Xh = X;
   if (K > 0) {
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
+      if (!(flags & QF_REUSE_W_HAT))
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
       Wh = w.w_hat;
     }
     if (a_amax_out) {
@@ -144,7 +145,8 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
       if (cudaError_t e = launch_amax_to_float(w.header + 6, a_amax_out, st)) return cu(e);
     }
     if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
-      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      if (!(flags & QF_REUSE_X_HAT))
+        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
       Xh = w.x_hat;
     }
   }
@@ -187,7 +189,8 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && wq == QF_FMT_MXFP4 && gemm_can_fuse(g);
     const void* Wh = W;
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
+      if (!(flags & QF_REUSE_W_HAT))
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
       Wh = w.w_hat;
     }
     g.B = Wh;
@@ -207,7 +210,8 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && aq == QF_FMT_MXFP4 && gemm_can_fuse(g);
     const void* Xh = X;
     if (aq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+      if (!(flags & QF_REUSE_X_HAT))
+        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
       Xh = w.x_hat;
     }
     g.B = Xh;

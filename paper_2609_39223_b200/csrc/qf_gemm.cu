@@ -1017,8 +1017,14 @@ template <bool A_MN, bool B_MN, typename OutT>
 cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
                      cudaStream_t st) {
   auto kern = gemm_kernel<A_MN, B_MN, OutT>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  if (e != cudaSuccess) return e;
+  static bool configured[64] = {false};           // per device: the attribute is a per-context property of the kernel
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
   kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, tmC, kp);
   return cudaGetLastError();
 }
@@ -1027,8 +1033,14 @@ template <bool A_MN, bool B_MN, typename OutT, int FUSE>
 cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
                           cudaStream_t st) {
   auto kern = gemm_pair_kernel<A_MN, B_MN, OutT, FUSE>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
-  if (e != cudaSuccess) return e;
+  static bool configured[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
   kern<<<grid, FUSE ? NUM_THREADS_FUSED : NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);   // cluster shape (2,1,1) is a kernel attribute
   return cudaGetLastError();
 }

@@ -329,3 +329,17 @@ def test_grouped_nvfp4_weights_have_one_tensor_scale_per_expert():
     _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
     with pytest.raises(api.QfError):          # the per-expert scale array is required
         api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NONE)
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NVFP4, api.FMT_NVFP4), (api.FMT_Q4_K, api.FMT_NONE)])
+def test_backward_can_reuse_the_forwards_quantized_copies(wq, aq):
+    M, N, K = 384, 520, 1024
+    c = synth.linear_case(M, N, K, seed=31, outlier_channels=2)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    dx0, dw0 = api.qf_fq_linear_bwd(dY, X, W, wq, aq)                      # recomputes W_hat and X_hat (the default)
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    wts = torch.zeros(1, device="cuda"); ats = torch.zeros(1, device="cuda")
+    api.qf_fq_linear_fwd(X, W, wq, aq, ws=ws, w_tscale=wts, a_tscale=ats)
+    dx1, dw1 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, ws=ws, w_tscale=wts, a_tscale=ats,
+                                    flags=api.REUSE_W_HAT | api.REUSE_X_HAT)
+    assert torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
