@@ -105,6 +105,20 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
                    void* codes, void* scales, float* tensor_scale, uint32_t flags, void* workspace,
                    size_t workspace_bytes, void* stream);
 
+/* LoRA-QAD weight path (Eq. qad-lora, Eq. export-lora): quantize-dequantize the MERGED weight
+ *     W_hat = Q^-1(Q(W + lora_scale * B A)),
+ * with W [rows, cols] BF16 (the frozen base), B [rows, rank] BF16 and A [rank, cols] BF16. The merge is
+ * done on the fly inside the quantizer kernels (and inside the amax pre-pass for NVFP4): the merged
+ * tensor is never written to memory, which is what lets a mixture-of-experts layer merge and quantize
+ * one expert after another without holding merged weights. Arithmetic of the merge, fixed so that results
+ * are reproducible: per element acc = W in FP32, then acc = fma(lora_scale * B[n,r], A[r,k], acc) for
+ * r = 0 .. rank-1 in that order (each step rounded once), then one rounding to BF16; the quantizer then
+ * sees that BF16 value. rank = 0 is qf_qdq. Other arguments as qf_qdq. A must be 16-byte aligned.
+ * To run the layer on the result, pass out_bf16 to the linear calls with wq_fmt = QF_FMT_NONE. */
+qf_status_t qf_qdq_lora(qf_format_t fmt, const void* W, const void* B, const void* A, int rank, float lora_scale,
+                        int64_t rows, int64_t cols, void* out_bf16, void* codes, void* scales, float* tensor_scale,
+                        uint32_t flags, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Q^-1 alone (Eq. nvfp4-dequant / Eq. mxfp4-dequant / Eq. q4k-dequant): codes + scales (+ tensor scale)
  * -> BF16 [rows, cols]. Layouts as in qf_qdq. */
 qf_status_t qf_dequant(qf_format_t fmt, const void* codes, const void* scales, const float* tensor_scale,

@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.orc_matmul_wgrad.restype = None
         L.orc_matmul_wgrad.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int64, c.c_int64,
                                        c.c_void_p, c.c_int64, c.c_void_p]
+        L.orc_lora_merge.restype = None
+        L.orc_lora_merge.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64, c.c_int64, c.c_float, c.c_void_p]
         _lib = L
     return _lib
 
@@ -255,3 +257,21 @@ def swizzle_block_scales(scales: np.ndarray) -> np.ndarray:
             ri = r % 128
             out[tile * 512 + (ri % 32) * 16 + (ri // 32) * 4 + c % 4] = scales[r, c]
     return out
+
+
+# ---- LoRA merge ahead of the quantizer (Eq. qad-lora) -----------------------------------------------
+
+def lora_merge(w, b, a, scale: float = 1.0) -> np.ndarray:
+    """bf16(W + scale * B A): FP32 accumulation over the rank in order, one fused multiply-add per step."""
+    w, b, a = _bf16_arr(w), _bf16_arr(b), _bf16_arr(a)
+    rows, cols = w.shape
+    rank = a.shape[0]
+    assert b.shape == (rows, rank) and a.shape == (rank, cols)
+    out = np.empty_like(w)
+    lib().orc_lora_merge(_p(w), _p(b), _p(a), rows, cols, rank, float(scale), _p(out))
+    return out
+
+
+def qdq_lora(fmt: int, w, b, a, scale: float = 1.0, tensor_scale: float | None = None):
+    """Q^-1(Q(W + scale * B A)): the quantizer applied to the merged weight."""
+    return qdq(fmt, lora_merge(w, b, a, scale), tensor_scale)

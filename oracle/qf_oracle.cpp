@@ -382,6 +382,23 @@ int orc_dequant(int fmt, const uint8_t* codes, const uint8_t* scales, const floa
     return 0;
 }
 
+// LoRA merge ahead of the quantizer (Eq. qad-lora): merged = bf16(W + scale * B A), W [rows, cols],
+// B [rows, rank], A [rank, cols]. FP32 accumulation in a fixed order, one fused multiply-add per rank
+// step (std::fmaf rounds once), then one rounding to BF16.
+void orc_lora_merge(const uint16_t* W, const uint16_t* B, const uint16_t* A, int64_t rows, int64_t cols, int64_t rank,
+                    float scale, uint16_t* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < rows; ++n)
+    for (int64_t k = 0; k < cols; ++k) {
+      float acc = bf16_to_f32(W[n * cols + k]);
+      for (int64_t r = 0; r < rank; ++r) {
+        const float b = scale * bf16_to_f32(B[n * rank + r]);
+        acc = std::fmaf(b, bf16_to_f32(A[r * cols + k]), acc);
+      }
+      out[n * cols + k] = f32_to_bf16(acc);
+    }
+}
+
 // Y[m,n] = sum_k Xh[m,k] * Wh[n,k]   (Eq. fakequant: O = W_hat A_hat, written for row-major
 // activations [M,K] and weights [N,K]). BF16 operands, FP64 accumulation, FP32 result.
 void orc_matmul_fwd(const uint16_t* Xh, const uint16_t* Wh, int64_t M, int64_t N, int64_t K, float* Y) {

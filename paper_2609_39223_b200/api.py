@@ -26,7 +26,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libqf.so"
 EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
-    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack", "qf_nvfp4_tensor_scale",
+    "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack", "qf_nvfp4_tensor_scale", "qf_qdq_lora",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 LAYOUT_GGUF_Q4_K, LAYOUT_FP4_SWIZZLED_SCALES = 1, 2
@@ -81,6 +81,9 @@ def lib() -> ctypes.CDLL:
         L.qf_fq_linear_fwd_noalloc.restype = c_int
         L.qf_fq_linear_fwd_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64, c_int64, c_int, c_int,
                                                c_void_p, c_void_p, c_uint32, c_void_p]
+        L.qf_qdq_lora.restype = c_int
+        L.qf_qdq_lora.argtypes = [c_int, c_void_p, c_void_p, c_void_p, c_int, c_float, c_int64, c_int64, c_void_p, c_void_p,
+                                  c_void_p, c_void_p, c_uint32, c_void_p, c_size_t, c_void_p]
         L.qf_nvfp4_tensor_scale.restype = c_int
         L.qf_nvfp4_tensor_scale.argtypes = [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_uint32, c_void_p]
         L.qf_pack_bytes.restype = c_size_t
@@ -330,3 +333,26 @@ def qf_nvfp4_tensor_scale(tensors, amax_state: torch.Tensor, *, running: bool = 
     _check(lib().qf_nvfp4_tensor_scale(ptrs, sizes, n, _ptr(amax_state), _ptr(scale), AMAX_RUNNING if running else 0, _stream()),
            "qf_nvfp4_tensor_scale")
     return scale
+
+
+def qf_qdq_lora(fmt: int, W: torch.Tensor, B: torch.Tensor, A: torch.Tensor, lora_scale: float = 1.0, *, tensor_scale=None,
+                ws=None):
+    """Quantize-dequantize of the merged weight W + lora_scale * B @ A without materialising the merge."""
+    W, B, A = _bf16(W, "W"), _bf16(B, "B"), _bf16(A, "A")
+    rows, cols = W.shape
+    rank = A.shape[0]
+    dev = W.device
+    out = torch.empty_like(W)
+    codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
+    scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=dev)
+    flags, ts = 0, None
+    if fmt == FMT_NVFP4:
+        if tensor_scale is not None:
+            ts, flags = tensor_scale, TENSOR_SCALE_GIVEN
+        else:
+            ts = torch.empty(1, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(OP_QDQ, rows, 0, cols, device=dev)
+    _check(lib().qf_qdq_lora(fmt, _ptr(W), _ptr(B), _ptr(A), rank, float(lora_scale), rows, cols, _ptr(out), _ptr(codes),
+                             _ptr(scales), _ptr(ts), flags, _ptr(ws), ws.numel(), _stream()), "qf_qdq_lora")
+    return {"out": out, "codes": codes, "scales": scales, "tensor_scale": ts}

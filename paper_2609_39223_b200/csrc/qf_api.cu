@@ -304,6 +304,50 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
   return cu(launch_qdq(q, st));
 }
 
+qf_status_t qf_qdq_lora(qf_format_t fmt, const void* W, const void* B, const void* A, int rank, float lora_scale, int64_t rows,
+                        int64_t cols, void* out_bf16, void* codes, void* scales, float* tensor_scale, uint32_t flags,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  if (!valid_fmt(fmt, false)) return QF_ERR_FORMAT;
+  if (rows < 0 || cols < 0 || cols % block_of(fmt) || rank < 0 || rank > 1024) return QF_ERR_SHAPE;
+  const bool empty = rows == 0 || cols == 0;
+  if (!empty && (!W || (rank > 0 && (!B || !A)))) return QF_ERR_NULL;
+  if (!empty && !out_bf16 && !codes && !scales) return QF_ERR_NULL;
+  if (fmt == QF_FMT_NVFP4 && !tensor_scale) return QF_ERR_NULL;
+  if (!aligned16(W) || !aligned16(A) || (out_bf16 && !aligned16(out_bf16)) || (codes && !aligned16(codes)) ||
+      (scales && !aligned16(scales)))
+    return QF_ERR_ALIGN;
+  if (B && (reinterpret_cast<uintptr_t>(B) & 1u)) return QF_ERR_ALIGN;
+  const bool need_amax = fmt == QF_FMT_NVFP4 && !(flags & QF_TENSOR_SCALE_GIVEN);
+  if (need_amax) {
+    if (!workspace || workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QF_ERR_ALIGN;
+  }
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  QdqArgs q{};
+  q.fmt = fmt;
+  q.in = W;
+  q.rows = rows;
+  q.cols = cols;
+  q.out = out_bf16;
+  q.codes = codes;
+  q.scales = scales;
+  q.lora_B = B;
+  q.lora_A = A;
+  q.lora_rank = empty ? 0 : rank;
+  q.lora_scale = lora_scale;
+  if (fmt == QF_FMT_NVFP4) {
+    if (need_amax) {
+      uint32_t* header = static_cast<uint32_t*>(workspace);
+      if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
+      q.tscale_out = tensor_scale;
+      return cu(launch_qdq_nvfp4_derive(q, header, kWsAmaxW, st));
+    }
+    q.tscale_in = tensor_scale;
+  }
+  return cu(launch_qdq(q, st));
+}
+
 qf_status_t qf_dequant(qf_format_t fmt, const void* codes, const void* scales, const float* tensor_scale, int64_t rows,
                        int64_t cols, void* out_bf16, void* stream) {
   if (!valid_fmt(fmt, false)) return QF_ERR_FORMAT;

@@ -125,6 +125,11 @@ struct QdqArgs {
   float* tscale_out;             // NVFP4: where the derived scale is written (nullable)
   bool reverse;                  // walk the tensor back to front (after an amax pass: L2 holds the tail)
   int groups;                    // NVFP4: > 1 = that many equal tensors back to back, each with its own tensor scale
+  // LoRA merge ahead of the quantizer (lora_rank > 0): the input is W + lora_scale * B A, formed on the fly
+  const void* lora_B;            // [rows, rank] BF16
+  const void* lora_A;            // [rank, cols] BF16
+  int lora_rank;
+  float lora_scale;
 };
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);

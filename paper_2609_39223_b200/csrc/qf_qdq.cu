@@ -16,6 +16,42 @@ constexpr int kThreads = 256;
 
 __device__ __forceinline__ uint4 ld_chunk(const uint4* p) { return __ldg(p); }
 
+// Where a kernel's 16-byte input chunks come from. PlainLoader reads the tensor. LoraLoader produces
+// the chunk of the merged weight W + s * B A (Eq. qad-lora) on the fly, so the merged tensor is never
+// written to memory: per element acc = W; acc = fma(s * B[n,r], A[r,k], acc) for r = 0 .. rank-1 in FP32
+// (one rounding per step, in this order), then one rounding to BF16.
+struct PlainLoader {
+  const uint4* in;
+  __device__ __forceinline__ uint4 chunk(int64_t c) const { return __ldg(in + c); }
+  __device__ __forceinline__ PlainLoader slice(int64_t chunks) const { return PlainLoader{in + chunks}; }
+};
+
+struct LoraLoader {
+  const uint4* W;                 // [rows, cols] BF16
+  const __nv_bfloat16* B;         // [rows, rank] BF16
+  const uint4* A;                 // [rank, cols] BF16
+  int rank;
+  float scale;
+  int64_t chunks_per_row;         // cols / 8
+  __device__ __forceinline__ uint4 chunk(int64_t c) const {
+    const int64_t row = c / chunks_per_row;
+    const int64_t kc = c - row * chunks_per_row;
+    const uint4 w = __ldg(W + c);
+    float acc[8] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y), bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
+    const __nv_bfloat16* brow = B + row * rank;
+    for (int r = 0; r < rank; ++r) {
+      const float b = __fmul_rn(scale, __bfloat162float(brow[r]));
+      const uint4 a = __ldg(A + r * chunks_per_row + kc);
+      acc[0] = __fmaf_rn(b, bf16_lo(a.x), acc[0]); acc[1] = __fmaf_rn(b, bf16_hi(a.x), acc[1]);
+      acc[2] = __fmaf_rn(b, bf16_lo(a.y), acc[2]); acc[3] = __fmaf_rn(b, bf16_hi(a.y), acc[3]);
+      acc[4] = __fmaf_rn(b, bf16_lo(a.z), acc[4]); acc[5] = __fmaf_rn(b, bf16_hi(a.z), acc[5]);
+      acc[6] = __fmaf_rn(b, bf16_lo(a.w), acc[6]); acc[7] = __fmaf_rn(b, bf16_hi(a.w), acc[7]);
+    }
+    return make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+  }
+  __device__ __forceinline__ LoraLoader slice(int64_t) const { return *this; }     // grouped slices are not combined with LoRA
+};
+
 // max |x| over the 8 BF16 values of a chunk, as BF16 bits (sign clear)
 __device__ __forceinline__ uint32_t chunk_amax_bits(const uint4& v) { return chunk8_amax_bits(v.x, v.y, v.z, v.w); }
 
@@ -23,21 +59,21 @@ __device__ __forceinline__ uint32_t chunk_amax_bits(const uint4& v) { return chu
 // tensor amax
 // ---------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t nchunks,
+template <typename Loader>
+__global__ void __launch_bounds__(kThreads) amax_kernel(Loader src, int64_t nchunks,
                                                         const __nv_bfloat16* __restrict__ tail, int ntail,
                                                         uint32_t* __restrict__ amax_bits) {
   // gridDim.y > 1: one tensor per y-slice (the experts of a grouped layer), nchunks chunks each
-  in += static_cast<int64_t>(blockIdx.y) * nchunks;
+  const Loader in = src.slice(static_cast<int64_t>(blockIdx.y) * nchunks);
   amax_bits += blockIdx.y;
   uint32_t m = 0;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
   int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
   for (; i + 3 * stride < nchunks; i += 4 * stride) {
-    uint4 a = ld_chunk(in + i), b = ld_chunk(in + i + stride), c = ld_chunk(in + i + 2 * stride),
-          d = ld_chunk(in + i + 3 * stride);
+    uint4 a = in.chunk(i), b = in.chunk(i + stride), c = in.chunk(i + 2 * stride), d = in.chunk(i + 3 * stride);
     m = max(m, max(max(chunk_amax_bits(a), chunk_amax_bits(b)), max(chunk_amax_bits(c), chunk_amax_bits(d))));
   }
-  for (; i < nchunks; i += stride) m = max(m, chunk_amax_bits(ld_chunk(in + i)));
+  for (; i < nchunks; i += stride) m = max(m, chunk_amax_bits(in.chunk(i)));
   if (blockIdx.x == 0 && threadIdx.x < ntail)
     m = max(m, static_cast<uint32_t>(__bfloat16_as_ushort(tail[threadIdx.x])) & 0x7FFFu);
   m = __reduce_max_sync(0xFFFFFFFFu, m);
@@ -190,17 +226,17 @@ __device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax
 
 constexpr int kUnitsPerThread = 2;
 
-template <int FMT>
-__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restrict__ in, int64_t nunits,
+template <int FMT, typename Loader>
+__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t nunits,
                                                            uint4* __restrict__ out, uint2* __restrict__ codes,
                                                            uint8_t* __restrict__ scales,
                                                            const float* __restrict__ tscale_in,
                                                            const uint32_t* __restrict__ amax_bits,
                                                            float* __restrict__ tscale_out, int reverse) {
   // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
+  const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
+  const Loader in = src.slice(2 * goff);
   {
-    const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
-    in += 2 * goff;
     if (out) out += 2 * goff;
     if (codes) codes += goff;
     if (scales) scales += FMT == QF_FMT_NVFP4 ? goff : goff / 2;
@@ -233,8 +269,8 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(const uint4* __restri
       // reverse: walk whole warps' worth of units from the end (block pairs of lanes stay adjacent)
       const int64_t i = reverse ? (nunits_up - 32 - (lin - lane)) + lane : lin;
       ok[u] = lin < nunits_up && i < nunits;      // lin past the end would map to a negative index in reverse
-      v[u][0] = ok[u] ? ld_chunk(in + 2 * i) : make_uint4(0, 0, 0, 0);
-      v[u][1] = ok[u] ? ld_chunk(in + 2 * i + 1) : make_uint4(0, 0, 0, 0);
+      v[u][0] = ok[u] ? in.chunk(2 * i) : make_uint4(0, 0, 0, 0);
+      v[u][1] = ok[u] ? in.chunk(2 * i + 1) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int u = 0; u < kUnitsPerThread; ++u) {
@@ -336,7 +372,8 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
   }
 }
 
-__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(const uint4* __restrict__ in, int64_t nsub,
+template <typename Loader>
+__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(Loader in, int64_t nsub,
                                                            uint4* __restrict__ out, uint4* __restrict__ codes,
                                                            uint4* __restrict__ scales) {
   const int lane = threadIdx.x & 31;
@@ -348,7 +385,7 @@ __global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(con
     uint32_t w[16];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const uint4 v = ok ? ld_chunk(in + 4 * i + k) : make_uint4(0, 0, 0, 0);
+      const uint4 v = ok ? in.chunk(4 * i + k) : make_uint4(0, 0, 0, 0);
       w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
     }
     __nv_bfloat162 mn = bits_bf2(w[0]), mx = bits_bf2(w[0]);
@@ -561,17 +598,22 @@ cudaError_t launch_amax_grouped(const void* in, int64_t n, int G, uint32_t* amax
   int gx = grid_for(nchunks, 4);
   const int cap = (kNumSMs * 8 + G - 1) / G;
   if (gx > cap) gx = cap < 1 ? 1 : cap;
-  amax_kernel<<<dim3(gx, G), kThreads, 0, st>>>(static_cast<const uint4*>(in), nchunks, nullptr, 0, amax_bits);
+  amax_kernel<PlainLoader><<<dim3(gx, G), kThreads, 0, st>>>(PlainLoader{static_cast<const uint4*>(in)}, nchunks, nullptr, 0, amax_bits);
   return cudaGetLastError();
 }
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st) {
   const int64_t nchunks = n / 8;
   const int ntail = static_cast<int>(n % 8);
-  amax_kernel<<<grid_for(nchunks, 4), kThreads, 0, st>>>(static_cast<const uint4*>(in), nchunks,
-                                                         static_cast<const __nv_bfloat16*>(in) + nchunks * 8, ntail,
-                                                         amax_bits);
+  amax_kernel<PlainLoader><<<grid_for(nchunks, 4), kThreads, 0, st>>>(PlainLoader{static_cast<const uint4*>(in)}, nchunks,
+                                                                      static_cast<const __nv_bfloat16*>(in) + nchunks * 8, ntail,
+                                                                      amax_bits);
   return cudaGetLastError();
+}
+
+static LoraLoader lora_loader(const QdqArgs& a) {
+  return LoraLoader{static_cast<const uint4*>(a.in), static_cast<const __nv_bfloat16*>(a.lora_B), static_cast<const uint4*>(a.lora_A),
+                    a.lora_rank, a.lora_scale, a.cols / 8};
 }
 
 cudaError_t launch_amax_to_scale(const uint32_t* amax_bits, float* scale, cudaStream_t st) {
@@ -584,29 +626,36 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
   return cudaGetLastError();
 }
 
-cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st) {
+template <typename Loader>
+static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStream_t st) {
   const int64_t nelem = a.rows * a.cols;
-  // an empty NVFP4 tensor still has a tensor scale to report (1.0): let one block write it
-  if (nelem == 0 && !(a.fmt == QF_FMT_NVFP4 && a.tscale_out)) return cudaSuccess;
-  const uint4* in = static_cast<const uint4*>(a.in);
   uint4* out = static_cast<uint4*>(a.out);
   if (a.fmt == QF_FMT_NVFP4) {
     const int slices = a.groups > 1 ? a.groups : 1;
     const int64_t nunits = nelem / 16 / slices;
     int gx = capped_grid(nunits, kUnitsPerThread, 16);
     if (slices > 1 && gx > (kNumSMs * 16 + slices - 1) / slices) gx = (kNumSMs * 16 + slices - 1) / slices;
-    qdq_fp4_kernel<QF_FMT_NVFP4><<<dim3(gx, slices), kThreads, 0, st>>>(
+    qdq_fp4_kernel<QF_FMT_NVFP4, Loader><<<dim3(gx, slices), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), a.tscale_in, a.amax_bits, a.tscale_out,
         a.reverse ? 1 : 0);
   } else if (a.fmt == QF_FMT_MXFP4) {
     const int64_t nunits = nelem / 16;
-    qdq_fp4_kernel<QF_FMT_MXFP4><<<capped_grid(nunits, kUnitsPerThread, 0), kThreads, 0, st>>>(
+    qdq_fp4_kernel<QF_FMT_MXFP4, Loader><<<capped_grid(nunits, kUnitsPerThread, 0), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr, 0);
   } else {
     const int64_t nsub = nelem / 32;
-    qdq_q4k_kernel<<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes), static_cast<uint4*>(a.scales));
+    qdq_q4k_kernel<Loader><<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes),
+                                                                          static_cast<uint4*>(a.scales));
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st) {
+  const int64_t nelem = a.rows * a.cols;
+  // an empty NVFP4 tensor still has a tensor scale to report (1.0): let one block write it
+  if (nelem == 0 && !(a.fmt == QF_FMT_NVFP4 && a.tscale_out)) return cudaSuccess;
+  if (a.lora_rank > 0) return launch_qdq_with(a, lora_loader(a), st);
+  return launch_qdq_with(a, PlainLoader{static_cast<const uint4*>(a.in)}, st);
 }
 
 // NVFP4 with a derived tensor scale: tensor amax, then quantize. The second pass walks the tensor
@@ -628,9 +677,16 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
     return launch_qdq(q, st);
   }
   uint32_t* amax_bits = header + amax_word;
-  if (cudaError_t e = launch_amax(a.in, a.rows * a.cols, amax_bits, st)) return e;
+  if (a.lora_rank > 0) {
+    // the absolute maximum is that of the merged weight, so the amax pass merges on the fly as well
+    const int64_t nchunks = a.rows * a.cols / 8;
+    if (nchunks > 0) amax_kernel<LoraLoader><<<grid_for(nchunks, 4), kThreads, 0, st>>>(lora_loader(a), nchunks, nullptr, 0, amax_bits);
+    if (cudaError_t e = cudaGetLastError()) return e;
+  } else {
+    if (cudaError_t e = launch_amax(a.in, a.rows * a.cols, amax_bits, st)) return e;
+    q.reverse = true;
+  }
   q.amax_bits = amax_bits;
-  q.reverse = true;
   return launch_qdq(q, st);
 }
 
