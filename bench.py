@@ -283,9 +283,11 @@ def run_ours(args):
     dX = torch.empty((M, K), dtype=torch.bfloat16, device=dev)
     dW = torch.empty((N, K), dtype=torch.float32, device=dev)
 
+    step_flags = api.FUSED_QDQ if args.in_kernel_qdq else 0
+
     def step():
-        api.qf_fq_linear_fwd(X, W, fmt, fmt, ws=ws, Y=Y)
-        api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, ws=ws, dX=dX, dW=dW)
+        api.qf_fq_linear_fwd(X, W, fmt, fmt, ws=ws, Y=Y, flags=step_flags)
+        api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, ws=ws, dX=dX, dW=dW, flags=step_flags)
 
     def barrier():
         replicas.barrier()
@@ -440,10 +442,11 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "wq_fmt": "mxfp4", "aq_fmt": "mxfp4", "M": M, "N": N, "K": K,
                        "outputs": "Y bf16, dX bf16, dW f32", "parallelism": f"replicas x{world}",
+                       "qdq": "inside the matmul kernel (QF_FUSED_QDQ)" if args.in_kernel_qdq else "materialised in the workspace (default)",
                        "l2": "inputs (369 MB) larger than L2; no flush"},
             "clocks": clocks,
             "e2e": e2e,
-            "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "gpu_launches": (3 if args.in_kernel_qdq else KERNELS_PER_STEP) * args.steps,
             "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel (tcgen05 cta_group::2 BF16, 256x256x64 tiles per CTA pair)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
                          # mean dram__bytes_read.sum + dram__bytes_write.sum per launch over the three matmuls of a
@@ -472,6 +475,8 @@ def main():
                     help="extra measurements beside the headline: roofline,qdq,e2e,cpu (default), configs = the other "
                          "named workloads (empty string: none)")
     ap.add_argument("--shape", default=None, help="M,N,K of a smaller case (profiler captures only)")
+    ap.add_argument("--in-kernel-qdq", action="store_true",
+                    help="run the step with QF_FUSED_QDQ (quantize the staged tiles inside the matmul kernel) instead of the default path")
     args = ap.parse_args()
     if args.shape:
         _set_shape(args.shape)

@@ -541,10 +541,11 @@ constexpr int B2_BYTES = (BN / 2) * BK * 2;     // 16 KB: this CTA's 128 rows of
 constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256 + 4 * (MAX_PAIR_GROUPS + 4);
 
-constexpr int TRANSFORM_WARPS = 8;                       // fused variant: warps that quantize-dequantize staged tiles
-constexpr int TRANSFORM_GROUPS = 4;                      // group g takes k-blocks g, g + 4, ...
+constexpr int TRANSFORM_WARPS = 16;                      // fused variant: warps that quantize-dequantize staged tiles
+constexpr int TRANSFORM_GROUPS = 4;                      // group g takes k-blocks g, g + 4, ... (must not exceed STAGES2)
 constexpr int WARPS_PER_GROUP = TRANSFORM_WARPS / TRANSFORM_GROUPS;
 constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * TRANSFORM_WARPS;
+static_assert(TRANSFORM_GROUPS <= 6, "more groups than pipeline stages would let a group wait on a stage two uses ahead");
 
 struct alignas(8) Barriers2 {
   uint64_t ready[STAGES2];      // fused variant, leader's copy: both CTAs' tiles have been quantized in place
@@ -870,7 +871,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t stage = it % STAGES2, phase = (it / STAGES2) & 1u;
         // one lane polls the barrier; the warp then proceeds together (the shuffles need all lanes)
         int got = 1;
-        if (lane == 0) got = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status) ? 1 : 0;
+        if (lane == 0) {
+          // A group may run ahead of the others. Before trusting full[stage] for its second and later uses,
+          // make sure the previous use of this stage has been consumed (its MMAs committed to empty[stage]);
+          // otherwise a parity wait could be satisfied by the phase of the previous use.
+          if (it >= STAGES2) got = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status) ? 1 : 0;
+          if (got) got = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, p.status) ? 1 : 0;
+        }
         got = __shfl_sync(0xFFFFFFFFu, got, 0);
         if (!got) { alive = false; break; }
         const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
