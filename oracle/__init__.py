@@ -64,7 +64,7 @@ def lib() -> ctypes.CDLL:
         L.orc_amax.argtypes = [c.c_void_p, c.c_int64]
         L.orc_qdq.restype = c.c_int
         L.orc_qdq.argtypes = [c.c_int, c.c_void_p, c.c_int64, c.c_int64, c.c_void_p, c.c_void_p,
-                              c.c_void_p, c.c_void_p, c.c_int]
+                              c.c_void_p, c.c_void_p, c.c_int, c.c_int]
         L.orc_dequant.restype = c.c_int
         L.orc_dequant.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int64, c.c_int64,
                                   c.c_void_p]
@@ -144,10 +144,12 @@ def scales_shape(fmt: int, rows: int, cols: int):
     return (rows, cols // BLOCK[fmt])
 
 
-def qdq(fmt: int, x, tensor_scale: float | None = None):
+def qdq(fmt: int, x, tensor_scale: float | None = None, mxfp4_noclip: bool = False):
     """Quantize-dequantize a BF16 [rows, cols] tensor. Returns a dict with ``out`` (uint16 BF16
     bits), ``codes`` (uint8, two 4-bit codes per byte), ``scales`` (uint8 metadata) and
-    ``tensor_scale`` (float32, NVFP4 only; given or derived from the tensor's absolute maximum)."""
+    ``tensor_scale`` (float32, NVFP4 only; given or derived from the tensor's absolute maximum).
+    ``mxfp4_noclip`` picks the MXFP4 block exponent as the smallest one under which the block
+    maximum does not saturate, instead of floor(log2 amax) - 2."""
     x = _bf16_arr(x)
     rows, cols = x.shape
     out = np.empty_like(x)
@@ -155,18 +157,18 @@ def qdq(fmt: int, x, tensor_scale: float | None = None):
     scales = np.empty(scales_shape(fmt, rows, cols), np.uint8)
     ts = np.array([0.0 if tensor_scale is None else tensor_scale], np.float32)
     rc = lib().orc_qdq(fmt, _p(x), rows, cols, _p(out), _p(codes), _p(scales), _p(ts),
-                       0 if tensor_scale is None else 1)
+                       0 if tensor_scale is None else 1, 1 if mxfp4_noclip else 0)
     if rc != 0:
         raise ValueError("orc_qdq: bad format or shape")
     return {"out": out, "codes": codes, "scales": scales,
             "tensor_scale": np.float32(ts[0]) if fmt == FMT_NVFP4 else None}
 
 
-def qdq_out(fmt: int, x, tensor_scale: float | None = None) -> np.ndarray:
+def qdq_out(fmt: int, x, tensor_scale: float | None = None, mxfp4_noclip: bool = False) -> np.ndarray:
     """X_hat only; ``fmt == FMT_NONE`` is the identity (an unquantized operand)."""
     if fmt == FMT_NONE:
         return _bf16_arr(x)
-    return qdq(fmt, x, tensor_scale)["out"]
+    return qdq(fmt, x, tensor_scale, mxfp4_noclip)["out"]
 
 
 def dequant(fmt: int, codes, scales, tensor_scale, rows: int, cols: int) -> np.ndarray:
@@ -216,16 +218,17 @@ def matmul_wgrad(dy, xh, n_idx=None) -> np.ndarray:
 
 # ---- the quantization-aware layer (Eq. fakequant) and its STE backward (Eq. ste) ---------------
 
-def fq_linear_fwd(x, w, wq_fmt: int, aq_fmt: int, w_tscale=None, a_tscale=None) -> np.ndarray:
+def fq_linear_fwd(x, w, wq_fmt: int, aq_fmt: int, w_tscale=None, a_tscale=None, mxfp4_noclip=False) -> np.ndarray:
     """Y = QDQ_a(X) . QDQ_w(W)^T with X [M,K], W [N,K]; returns float32 [M,N]."""
-    return matmul_fwd(qdq_out(aq_fmt, x, a_tscale), qdq_out(wq_fmt, w, w_tscale))
+    return matmul_fwd(qdq_out(aq_fmt, x, a_tscale, mxfp4_noclip), qdq_out(wq_fmt, w, w_tscale, mxfp4_noclip))
 
 
-def fq_linear_bwd(dy, x, w, wq_fmt: int, aq_fmt: int, w_tscale=None, a_tscale=None, n_idx=None):
+def fq_linear_bwd(dy, x, w, wq_fmt: int, aq_fmt: int, w_tscale=None, a_tscale=None, n_idx=None,
+                  mxfp4_noclip=False):
     """(dX, dW): dX = dY . QDQ_w(W), dW = dY^T . QDQ_a(X). The quantizers are treated as the
     identity in the backward pass; dY itself is never quantized."""
-    dx = matmul_dgrad(dy, qdq_out(wq_fmt, w, w_tscale))
-    dw = matmul_wgrad(dy, qdq_out(aq_fmt, x, a_tscale), n_idx)
+    dx = matmul_dgrad(dy, qdq_out(wq_fmt, w, w_tscale, mxfp4_noclip))
+    dw = matmul_wgrad(dy, qdq_out(aq_fmt, x, a_tscale, mxfp4_noclip), n_idx)
     return dx, dw
 
 

@@ -169,10 +169,12 @@ void nvfp4_row(const uint16_t* x, int64_t cols, float s_t, uint16_t* out, uint8_
 
 // ---------------------------------------------------------------------------------------------
 // MXFP4 (Eq. mxfp4, Eq. mxfp4-dequant): E2M1 codes, blocks of 32, power-of-two E8M0 block scale.
-// x_hat_i = 2^{p_b} * C_i.  Scale rule: p = floor(log2 amax) - 2, clamped to [-127, 127].
+// x_hat_i = 2^{p_b} * C_i.  Scale rule: p = floor(log2 amax) - 2, clamped to [-127, 127]; block
+// maxima in (6, 8) * 2^p then saturate at 6 * 2^p. The paper does not fix the rule; the variant
+// `noclip` takes instead the smallest p in [-127, 127] with amax <= 6 * 2^p, so nothing saturates.
 // ---------------------------------------------------------------------------------------------
 
-void mxfp4_row(const uint16_t* x, int64_t cols, uint16_t* out, uint8_t* codes, uint8_t* scales) {
+void mxfp4_row(const uint16_t* x, int64_t cols, uint16_t* out, uint8_t* codes, uint8_t* scales, bool noclip) {
     const int B = 32;
     for (int64_t b = 0; b < cols / B; ++b) {
         const uint16_t* xb = x + b * B;
@@ -191,6 +193,10 @@ void mxfp4_row(const uint16_t* x, int64_t cols, uint16_t* out, uint8_t* codes, u
             p = (e - 1) - 2;
             if (p < -127) p = -127;
             if (p > 127) p = 127;
+            if (noclip) {
+                p = -127;
+                while (p < 127 && static_cast<double>(amax_b) > 6.0 * std::ldexp(1.0, p)) ++p;
+            }
             float inv = exp2i(-p);
             for (int i = 0; i < B; ++i) c[i] = e2m1_encode(bf16_to_f32(xb[i]) * inv);
         }
@@ -312,9 +318,10 @@ float orc_amax(const uint16_t* x, int64_t n) { return tensor_amax(x, n); }
 
 // Quantize-dequantize of a row-major BF16 [rows, cols] tensor, blocks along cols.
 // out / codes / scales may be null. NVFP4: *tensor_scale is read when tscale_given != 0, otherwise
-// derived from the tensor's absolute maximum and written back. Returns 0, or -1 on a bad shape.
+// derived from the tensor's absolute maximum and written back. mxfp4_noclip != 0 selects the MXFP4
+// scale rule without saturation. Returns 0, or -1 on a bad shape.
 int orc_qdq(int fmt, const uint16_t* in, int64_t rows, int64_t cols, uint16_t* out, uint8_t* codes,
-            uint8_t* scales, float* tensor_scale, int tscale_given) {
+            uint8_t* scales, float* tensor_scale, int tscale_given, int mxfp4_noclip) {
     int block = fmt == ORC_FMT_NVFP4 ? 16 : fmt == ORC_FMT_MXFP4 ? 32 : fmt == ORC_FMT_Q4_K ? 256 : 0;
     if (block == 0 || rows < 0 || cols < 0 || cols % block) return -1;
     float s_t = 1.0f;
@@ -336,7 +343,7 @@ int orc_qdq(int fmt, const uint16_t* in, int64_t rows, int64_t cols, uint16_t* o
         uint8_t* c = codes ? codes + r * code_stride : nullptr;
         uint8_t* s = scales ? scales + r * scale_stride : nullptr;
         if (fmt == ORC_FMT_NVFP4) nvfp4_row(x, cols, s_t, o, c, s);
-        else if (fmt == ORC_FMT_MXFP4) mxfp4_row(x, cols, o, c, s);
+        else if (fmt == ORC_FMT_MXFP4) mxfp4_row(x, cols, o, c, s, mxfp4_noclip != 0);
         else q4k_row(x, cols, o, c, s);
     }
     return 0;

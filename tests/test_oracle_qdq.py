@@ -235,6 +235,63 @@ def test_mxfp4_zero_block_subnormals_and_extremes():
     assert 0xFF not in r["scales"]
 
 
+def test_mxfp4_noclip_worked_blocks():
+    for p, xs, want in _rows("mxfp4_noclip_worked.txt"):
+        x = np.zeros((1, 32), np.float32)
+        x[0, :len(xs)] = [float(v) for v in xs]
+        r = oracle.qdq(FMT_MXFP4, f32_to_bits(x), mxfp4_noclip=True)
+        assert int(r["scales"][0, 0]) - 127 == int(p[0])
+        np.testing.assert_array_equal(bits_to_f32(r["out"])[0, :len(want)], np.array([float(v) for v in want], np.float32))
+
+
+def test_mxfp4_noclip_rule_is_minimal_exponent_without_saturation():
+    rng = np.random.default_rng(29)
+    x = bits_to_f32(f32_to_bits(rng.normal(0, 1, (32, 512)) * np.exp(rng.uniform(-8, 8, (32, 1)))))
+    xb = f32_to_bits(x)
+    r0 = oracle.qdq(FMT_MXFP4, xb)
+    r1 = oracle.qdq(FMT_MXFP4, xb, mxfp4_noclip=True)
+    p0 = r0["scales"].astype(np.int64) - 127
+    p1 = r1["scales"].astype(np.int64) - 127
+    amax = np.abs(x.astype(np.float64)).reshape(32, -1, 32).max(-1)
+    # one step up exactly where the floor rule would saturate the block maximum
+    np.testing.assert_array_equal(p1 - p0, (amax > 6 * np.exp2(p0)).astype(np.int64))
+    assert 0 < (p1 != p0).mean() < 1
+    assert np.all(amax <= 6 * np.exp2(p1)) and np.all(amax > 6 * np.exp2(p1 - 1))      # smallest such exponent
+    # dequantization equation, and nearest grid point with nothing outside the grid's range
+    codes = unpack_nibbles(r1["codes"])
+    want = np.exp2(p1.astype(np.float64)).repeat(32, axis=1) * E2M1_VALUES[codes]
+    np.testing.assert_array_equal(bits_to_f32(r1["out"]).astype(np.float64), want)
+    np.testing.assert_array_equal(oracle.dequant(FMT_MXFP4, r1["codes"], r1["scales"], None, 32, 512), r1["out"])
+    v = x.astype(np.float64) / np.exp2(p1.astype(np.float64)).repeat(32, axis=1)
+    grid = np.array([0, .5, 1, 1.5, 2, 3, 4, 6], np.float64)
+    d = np.abs(np.abs(v)[..., None] - grid)
+    assert np.all(np.take_along_axis(d, (codes & 7)[..., None].astype(np.int64), -1)[..., 0] == d.min(-1))
+    assert np.abs(v).max() <= 6
+    assert np.all(np.abs(x - bits_to_f32(r1["out"])) <= np.exp2(p1.astype(np.float64)).repeat(32, axis=1))
+    # blocks the floor rule does not saturate are left as they were
+    same = (p1 == p0).repeat(32, axis=1)
+    np.testing.assert_array_equal(r1["out"][same], r0["out"][same])
+    np.testing.assert_array_equal(r1["codes"][same[:, ::2]], r0["codes"][same[:, ::2]])
+    # idempotent in value (a block whose maximum rounds to 3 * 2^p re-encodes one exponent lower)
+    np.testing.assert_array_equal(oracle.qdq(FMT_MXFP4, r1["out"], mxfp4_noclip=True)["out"], r1["out"])
+    np.testing.assert_array_equal(oracle.qdq(FMT_MXFP4, xb ^ 0x8000, mxfp4_noclip=True)["out"], r1["out"] ^ 0x8000)
+
+
+def test_mxfp4_noclip_extremes():
+    x = np.zeros((1, 160), np.float32)
+    x[0, 32:64] = 2.0 ** -133                     # smallest BF16 subnormal: the exponent clamps at -127
+    x[0, 64] = 2.9e38                             # 3.41 * 2^126 -> 3 * 2^126, finite
+    x[0, 96] = 6 * 2.0 ** -127                    # exactly 6 * 2^-127: lowest exponent, top code
+    x[0, 128] = -0.0
+    r = oracle.qdq(FMT_MXFP4, f32_to_bits(x), mxfp4_noclip=True)
+    assert list(r["scales"][0]) == [0, 0, 127 + 126, 0, 0]
+    out = bits_to_f32(r["out"])[0]
+    assert not r["out"][0, :64].any()
+    assert out[64] == 3 * 2.0 ** 126
+    assert out[96] == np.float32(6 * 2.0 ** -127)
+    assert r["out"][0, 128] == 0
+
+
 # ------------------------------------------------------------------------------------------
 # Q4_K
 # ------------------------------------------------------------------------------------------
