@@ -74,6 +74,13 @@ typedef enum {
                                       workspace first. Same results bit for bit. Applies to MXFP4 operands of
                                       non-grouped calls with M >= 256; anything else silently takes the default path. */
 
+#define QF_MXFP4_NO_CLIP 0x80u      /* qf_qdq, qf_qdq_lora and the linear calls: MXFP4 block exponent p = the smallest one
+                                      with amax <= 6 * 2^p (nothing saturates) instead of floor(log2 amax) - 2, under
+                                      which block maxima in (6, 8) * 2^p clamp to 6 * 2^p. The paper leaves the rule
+                                      open (Eq. mxfp4 only requires a power-of-two scale); the default follows the
+                                      shared-exponent convention of the MX formats. Blocks whose maximum exceeds
+                                      3.5 * 2^126 overflow to infinity under this rule. Other formats ignore the flag. */
+
 const char* qf_status_string(qf_status_t s);
 int qf_version(void);
 

@@ -18,6 +18,7 @@ OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 
 TENSOR_SCALE_GIVEN = 0x1
 W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x2, 0x4, 0x8, 0x10
 REUSE_W_HAT, REUSE_X_HAT = 0x20, 0x40
+MXFP4_NO_CLIP = 0x80
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 
@@ -152,9 +153,10 @@ def scales_shape(fmt: int, rows: int, cols: int):
 
 
 def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_scales=True, tensor_scale=None,
-           ws: torch.Tensor | None = None, out=None, codes=None, scales=None, ts_out=None):
+           ws: torch.Tensor | None = None, out=None, codes=None, scales=None, ts_out=None, flags: int = 0):
     """(C, theta) = Q(x), x_hat = Q^-1(C, theta). Returns dict(out, codes, scales, tensor_scale); the
-    tensor scale (NVFP4) is a 1-element float32 CUDA tensor, read if ``tensor_scale`` is given."""
+    tensor scale (NVFP4) is a 1-element float32 CUDA tensor, read if ``tensor_scale`` is given.
+    ``flags`` may carry MXFP4_NO_CLIP."""
     x = _bf16(x, "x")
     rows, cols = x.shape
     dev = x.device
@@ -164,7 +166,7 @@ def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_sc
         codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
     if want_scales and scales is None:
         scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=dev)
-    flags = 0
+    flags &= MXFP4_NO_CLIP
     ts = None
     if fmt == FMT_NVFP4:
         if tensor_scale is not None:
@@ -336,7 +338,7 @@ def qf_nvfp4_tensor_scale(tensors, amax_state: torch.Tensor, *, running: bool = 
 
 
 def qf_qdq_lora(fmt: int, W: torch.Tensor, B: torch.Tensor, A: torch.Tensor, lora_scale: float = 1.0, *, tensor_scale=None,
-                ws=None):
+                ws=None, flags: int = 0):
     """Quantize-dequantize of the merged weight W + lora_scale * B @ A without materialising the merge."""
     W, B, A = _bf16(W, "W"), _bf16(B, "B"), _bf16(A, "A")
     rows, cols = W.shape
@@ -345,10 +347,10 @@ def qf_qdq_lora(fmt: int, W: torch.Tensor, B: torch.Tensor, A: torch.Tensor, lor
     out = torch.empty_like(W)
     codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
     scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=dev)
-    flags, ts = 0, None
+    flags, ts = flags & MXFP4_NO_CLIP, None
     if fmt == FMT_NVFP4:
         if tensor_scale is not None:
-            ts, flags = tensor_scale, TENSOR_SCALE_GIVEN
+            ts, flags = tensor_scale, flags | TENSOR_SCALE_GIVEN
         else:
             ts = torch.empty(1, dtype=torch.float32, device=dev)
     if ws is None:

@@ -64,8 +64,9 @@ Workspace carve(void* ws, int64_t N, int64_t K, int64_t groups) {
 // array of `groups` floats (required).
 qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t cols, void* dst, float* tscale_user,
                              bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st,
-                             int groups = 1) {
+                             int groups = 1, bool mxfp4_noclip = false) {
   QdqArgs q{};
+  q.mxfp4_noclip = mxfp4_noclip;
   q.fmt = fmt;
   q.in = src;
   q.rows = rows;
@@ -126,6 +127,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   g.a_mn_major = false; g.b_mn_major = false;
   g.c_dtype = y_dtype;
   g.status_word = w.header + kWsStatus;
+  g.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
   if (grouped) {
     g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M;
   }
@@ -137,7 +139,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   if (K > 0) {
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
       if (!(flags & QF_REUSE_W_HAT))
-        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Wh = w.w_hat;
     }
     if (a_amax_out) {
@@ -146,7 +148,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
     }
     if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
       if (!(flags & QF_REUSE_X_HAT))
-        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Xh = w.x_hat;
     }
   }
@@ -185,12 +187,13 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.a_mn_major = false; g.b_mn_major = true;
     g.c_dtype = dx_dtype;
     g.status_word = w.header + kWsStatus;
+  g.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
     if (grouped) { g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M; }
     g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && wq == QF_FMT_MXFP4 && gemm_can_fuse(g);
     const void* Wh = W;
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
       if (!(flags & QF_REUSE_W_HAT))
-        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups))) return s;
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Wh = w.w_hat;
     }
     g.B = Wh;
@@ -206,12 +209,13 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.c_dtype = dw_dtype;
     g.accumulate = (flags & QF_ACCUMULATE_DW) != 0;
     g.status_word = w.header + kWsStatus;
+  g.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
     if (grouped) { g.group_mode = 2; g.group_offsets = offs; g.G = G; g.rows_padded = M; g.c_group_stride = N * K; }
     g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && aq == QF_FMT_MXFP4 && gemm_can_fuse(g);
     const void* Xh = X;
     if (aq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
       if (!(flags & QF_REUSE_X_HAT))
-        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st)) return s;
+        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Xh = w.x_hat;
     }
     g.B = Xh;
@@ -291,6 +295,7 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
   q.out = out_bf16;
   q.codes = codes;
   q.scales = scales;
+  q.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
   if (fmt == QF_FMT_NVFP4) {
     if (need_amax) {
       uint32_t* header = static_cast<uint32_t*>(workspace);
@@ -332,6 +337,7 @@ qf_status_t qf_qdq_lora(qf_format_t fmt, const void* W, const void* B, const voi
   q.out = out_bf16;
   q.codes = codes;
   q.scales = scales;
+  q.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
   q.lora_B = B;
   q.lora_A = A;
   q.lora_rank = empty ? 0 : rank;

@@ -64,9 +64,13 @@ __device__ __forceinline__ float e8m0_inv_scale(uint32_t code) { return __uint_a
 
 // MXFP4 block-scale code from the block's max |x| given as BF16 bits (sign clear):
 // p = floor(log2 amax) - 2 clamped to [-127, 127]; code = p + 127 = biased exponent - 2.
-__device__ __forceinline__ uint32_t mxfp4_scale_code(uint32_t amax_bf16_bits) {
-  int e = static_cast<int>(amax_bf16_bits >> 7);
-  return static_cast<uint32_t>(max(e - 2, 0));
+// noclip: the smallest p with amax <= 6 * 2^p instead. amax * 2^-p = 4 * (1 + mantissa / 128) under the
+// first rule, so that is one more exactly when the mantissa exceeds 64 (and the first rule did not clamp:
+// below biased exponent 2 the ratio is under 4 already).
+__device__ __forceinline__ uint32_t mxfp4_scale_code(uint32_t amax_bf16_bits, bool noclip) {
+  const int e = static_cast<int>(amax_bf16_bits >> 7);
+  const int bump = (noclip && e >= 2 && (amax_bf16_bits & 0x7Fu) > 0x40u) ? 1 : 0;
+  return static_cast<uint32_t>(max(e - 2, 0) + bump);
 }
 
 __device__ __forceinline__ float2 splat(float a) { return make_float2(a, a); }
@@ -124,6 +128,7 @@ struct QdqArgs {
   const uint32_t* amax_bits;     // NVFP4: tensor amax as FP32 bits (device) to derive it from
   float* tscale_out;             // NVFP4: where the derived scale is written (nullable)
   bool reverse;                  // walk the tensor back to front (after an amax pass: L2 holds the tail)
+  bool mxfp4_noclip;             // MXFP4: smallest block exponent without saturation (QF_MXFP4_NO_CLIP)
   int groups;                    // NVFP4: > 1 = that many equal tensors back to back, each with its own tensor scale
   // LoRA merge ahead of the quantizer (lora_rank > 0): the input is W + lora_scale * B A, formed on the fly
   const void* lora_B;            // [rows, rank] BF16
@@ -166,6 +171,7 @@ struct GemmArgs {
   int64_t rows_padded;           // mode 1: total rows of A / C; mode 2: total contraction rows
   uint32_t* status_word;         // device word receiving QF_ERR_TIMEOUT if a wait expires
   bool fuse_a_mxfp4, fuse_b_mxfp4;   // apply the MXFP4 quantize-dequantize to the staged tiles inside the kernel
+  bool mxfp4_noclip;                 // scale rule of that in-kernel quantizer (QF_MXFP4_NO_CLIP)
 };
 
 cudaError_t launch_pack_q4k(const void* codes, const void* scales, int64_t nsb, void* records, bool unpack, void* codes_out,

@@ -60,6 +60,7 @@ struct KParams {
   int64_t b_group_rows;      // mode 1: rows one group occupies in B's 2-D tensor map
   int64_t c_group_stride;    // mode 2: elements between per-group outputs
   uint32_t* status;
+  int mxfp4_noclip;          // scale rule of the in-kernel MXFP4 quantizer
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -674,7 +675,7 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
 // 512-byte span (bank-conflict free); the four lanes of a block combine their maxima by shuffles.
 // One batch: PER chunks per lane, loads first, then shuffles, then independent arithmetic chains, then stores.
 template <int PER>
-__device__ __forceinline__ void mxfp4_transform_batch(uint32_t slab) {
+__device__ __forceinline__ void mxfp4_transform_batch(uint32_t slab, bool noclip) {
   uint4 v[PER];
   uint32_t m[PER];
 #pragma unroll
@@ -687,7 +688,7 @@ __device__ __forceinline__ void mxfp4_transform_batch(uint32_t slab) {
   for (int i = 0; i < PER; ++i) m[i] = max(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], 2));
 #pragma unroll
   for (int i = 0; i < PER; ++i) {
-    const uint32_t code = mxfp4_scale_code(m[i]);
+    const uint32_t code = mxfp4_scale_code(m[i], noclip);
     const uint32_t dst = slab + static_cast<uint32_t>(i) * 512u;
     if (mxfp4_bf16_path_ok(code)) {
       // conversion-free rounding in packed BF16 arithmetic (the common case)
@@ -708,13 +709,13 @@ __device__ __forceinline__ void mxfp4_transform_batch(uint32_t slab) {
 // each warp owns a contiguous slab and walks it in batches of four chunks per lane (512 bytes per warp
 // per load instruction: bank-conflict free, and every aligned group of four lanes holds one 32-element block).
 template <int NCHUNKS>
-__device__ __forceinline__ void mxfp4_transform_tile(uint32_t base, int warp_in_group, int lane) {
+__device__ __forceinline__ void mxfp4_transform_tile(uint32_t base, int warp_in_group, int lane, bool noclip) {
   constexpr int PER_WARP = NCHUNKS / WARPS_PER_GROUP;          // chunks per warp
   constexpr int BATCH = 4;
   static_assert(PER_WARP % (32 * BATCH) == 0, "tile must split evenly");
   const uint32_t slab = base + static_cast<uint32_t>(warp_in_group * PER_WARP + lane) * 16u;
 #pragma unroll 1
-  for (int b = 0; b < PER_WARP / (32 * BATCH); ++b) mxfp4_transform_batch<BATCH>(slab + static_cast<uint32_t>(b) * (32u * BATCH * 16u));
+  for (int b = 0; b < PER_WARP / (32 * BATCH); ++b) mxfp4_transform_batch<BATCH>(slab + static_cast<uint32_t>(b) * (32u * BATCH * 16u), noclip);
 }
 
 // FUSE: bit 0 = quantize-dequantize the staged A tile (MXFP4), bit 1 = the staged B tile. With FUSE != 0
@@ -881,8 +882,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         got = __shfl_sync(0xFFFFFFFFu, got, 0);
         if (!got) { alive = false; break; }
         const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
-        if (FUSE & 1) mxfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane);
-        if (FUSE & 2) mxfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane);
+        if (FUSE & 1) mxfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane, p.mxfp4_noclip != 0);
+        if (FUSE & 2) mxfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane, p.mxfp4_noclip != 0);
         fence_async_smem();                          // make the generic-proxy writes visible to the tensor core
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->ready[stage]), 0));
@@ -1103,6 +1104,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.c_dtype = a.c_dtype;
   kp.accumulate = a.accumulate ? 1 : 0;
   kp.status = a.status_word;
+  kp.mxfp4_noclip = a.mxfp4_noclip ? 1 : 0;
   kp.group_mode = a.group_mode;
   kp.G = a.G;
   kp.offs = a.group_offsets;
@@ -1168,6 +1170,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   kp.offs = a.group_offsets;
   kp.c_group_stride = a.c_group_stride;
   kp.status = a.status_word;
+  kp.mxfp4_noclip = 0;
   const int64_t a_rows_total = a.group_mode == 1 ? a.rows_padded : a.Mo;   // rows of A (and of C) in mode 1
   kp.tiles_m = static_cast<int>((a_rows_total + BM - 1) / BM);
   kp.tiles_n = static_cast<int>((a.No + BN - 1) / BN);

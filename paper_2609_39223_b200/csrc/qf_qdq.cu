@@ -161,8 +161,9 @@ struct UnitOut {
 };
 
 // MXFP4: x_hat = 2^p * C with p = floor(log2 amax_block) - 2 (Eq. mxfp4-dequant). All products exact.
-__device__ __forceinline__ UnitOut mxfp4_unit(const uint32_t (&w)[8], uint32_t block_amax_bits, uint32_t& scale_code) {
-  scale_code = mxfp4_scale_code(block_amax_bits);
+__device__ __forceinline__ UnitOut mxfp4_unit(const uint32_t (&w)[8], uint32_t block_amax_bits, bool noclip,
+                                              uint32_t& scale_code) {
+  scale_code = mxfp4_scale_code(block_amax_bits, noclip);
   const float2 inv = splat(e8m0_inv_scale(scale_code));
   const float2 sc = splat(e8m0_scale(scale_code));
   const uint32_t keep = block_amax_bits == 0 ? 0u : 0xFFu;       // an all-zero block drops the sign of -0
@@ -232,7 +233,9 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
                                                            uint8_t* __restrict__ scales,
                                                            const float* __restrict__ tscale_in,
                                                            const uint32_t* __restrict__ amax_bits,
-                                                           float* __restrict__ tscale_out, int reverse) {
+                                                           float* __restrict__ tscale_out, int opts) {
+  const bool reverse = (opts & 1) != 0;       // walk back to front
+  const bool noclip = (opts & 2) != 0;        // MXFP4 scale rule without saturation
   // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
   const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
   const Loader in = src.slice(2 * goff);
@@ -283,7 +286,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
       UnitOut r;
       if (FMT == QF_FMT_MXFP4) {
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-        r = mxfp4_unit(w, m, scale_code);
+        r = mxfp4_unit(w, m, noclip, scale_code);
       } else {
         const float amax_b = __uint_as_float(m << 16);
         // quotients near the bottom of the FP32 range take the IEEE divide (warp-uniform choice)
@@ -641,7 +644,8 @@ static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStrea
   } else if (a.fmt == QF_FMT_MXFP4) {
     const int64_t nunits = nelem / 16;
     qdq_fp4_kernel<QF_FMT_MXFP4, Loader><<<capped_grid(nunits, kUnitsPerThread, 0), kThreads, 0, st>>>(
-        in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr, 0);
+        in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr,
+        a.mxfp4_noclip ? 2 : 0);
   } else {
     const int64_t nsub = nelem / 32;
     qdq_q4k_kernel<Loader><<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes),

@@ -248,6 +248,30 @@ def test_in_kernel_mxfp4_quantization_is_bitwise_the_workspace_path(wq, aq, M, N
     _close(y1, oracle.fq_linear_fwd(torch_to_bits(c.X), torch_to_bits(c.W), wq, aq), "Y fused")
 
 
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_MXFP4, api.FMT_NONE)])
+@pytest.mark.parametrize("M,N,K", [(200, 264, 768), (520, 776, 1024)])
+def test_mxfp4_scale_rule_without_saturation_through_the_layer(wq, aq, M, N, K):
+    """QF_MXFP4_NO_CLIP reaches both operands' quantizers, in the workspace path and in the in-kernel
+    one (bitwise the same again), forward and backward, and matches the oracle under the same rule."""
+    c = synth.linear_case(M, N, K, seed=3 * M + K, outlier_channels=4)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    xb, wb, dyb = torch_to_bits(c.X), torch_to_bits(c.W), torch_to_bits(c.dY)
+    f = api.MXFP4_NO_CLIP
+    y0 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32, flags=f)
+    dx0, dw0 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, flags=f)
+    _close(y0, oracle.fq_linear_fwd(xb, wb, wq, aq, mxfp4_noclip=True), "Y")
+    dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, wq, aq, mxfp4_noclip=True)
+    _close(dx0, dx_ref, "dX")
+    _close(dw0, dw_ref, "dW")
+    # the rule matters: the default rule's output differs
+    assert not torch.equal(y0, api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32))
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    y1 = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32, flags=f | api.FUSED_QDQ, ws=ws)
+    dx1, dw1 = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, flags=f | api.FUSED_QDQ, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
     status word and leave the context usable (no trap, no hang)."""

@@ -12,12 +12,12 @@ pytestmark = pytest.mark.gpu
 FMTS = [(api.FMT_NVFP4, "nvfp4"), (api.FMT_MXFP4, "mxfp4"), (api.FMT_Q4_K, "q4_k")]
 
 
-def _compare(fmt, xbits, tensor_scale=None):
+def _compare(fmt, xbits, tensor_scale=None, noclip=False):
     x = bits_to_torch(xbits, "cuda")
     ts = None if tensor_scale is None else torch.tensor([tensor_scale], dtype=torch.float32, device="cuda")
-    g = api.qf_qdq(fmt, x, tensor_scale=ts)
+    g = api.qf_qdq(fmt, x, tensor_scale=ts, flags=api.MXFP4_NO_CLIP if noclip else 0)
     torch.cuda.synchronize()
-    o = oracle.qdq(fmt, xbits, tensor_scale)
+    o = oracle.qdq(fmt, xbits, tensor_scale, mxfp4_noclip=noclip)
     np.testing.assert_array_equal(torch_to_bits(g["out"]), o["out"])
     np.testing.assert_array_equal(g["codes"].cpu().numpy(), o["codes"])
     np.testing.assert_array_equal(g["scales"].cpu().numpy(), o["scales"])
@@ -115,6 +115,42 @@ def test_mxfp4_ties_clipping_subnormals_extremes():
     x[2, :] = 0.02001953125
     x[3, 5] = -0.0
     _compare(api.FMT_MXFP4, f32_to_bits(x))
+
+
+@pytest.mark.parametrize("noclip", [False, True])
+def test_mxfp4_every_bf16_value_as_block_maximum(noclip):
+    """Both scale rules, with each of the 32640 finite positive BF16 values in turn as a block's
+    maximum (the rule is a function of that value alone); the other elements are fractions of it."""
+    amax = np.arange(1, 0x7F80, dtype=np.uint16)
+    rng = np.random.default_rng(41)
+    frac = rng.uniform(-1, 1, (amax.size, 32)).astype(np.float32)
+    frac[:, 7] = 1.0
+    x = f32_to_bits(frac * bits_to_f32(amax)[:, None])
+    x[:, 7] = amax                                                     # exact, whatever the product rounded to
+    pad = (-amax.size) % 8
+    x = np.concatenate([x, np.zeros((pad, 32), np.uint16)]).reshape(-1, 256)
+    g, o = _compare(api.FMT_MXFP4, x, noclip=noclip)
+    if noclip:
+        p0 = oracle.qdq(api.FMT_MXFP4, x)["scales"].astype(int)
+        assert set(np.unique(o["scales"].astype(int) - p0)) == {0, 1}
+
+
+def test_mxfp4_noclip_random_ragged_and_worked_blocks():
+    for shape, seed in [((37, 768), 5), ((129, 2304), 6), ((3, 64), 7)]:
+        _compare(api.FMT_MXFP4, torch_to_bits(synth.randn_bf16(shape, 1.0, seed)), noclip=True)
+    x = np.zeros((2, 128), np.float32)
+    x[0, :8] = [7, 5, 2.5, 3.5, 0.25, 0.75, 1.25, 1.75]
+    x[0, 32:35] = [6, 0.25, -1.75]
+    x[0, 64:68] = [6.03125, -6.03125, 1, 0.5]
+    x[1, :32] = 2.0 ** -133
+    x[1, 64] = 2.9e38
+    x[1, 96] = 6 * 2.0 ** -127
+    g, o = _compare(api.FMT_MXFP4, f32_to_bits(x), noclip=True)
+    assert list(bits_to_f32(torch_to_bits(g["out"]))[0, :8]) == [8, 4, 2, 4, 0, 1, 1, 2]
+    # the flag leaves the other formats alone
+    xb = torch_to_bits(synth.randn_bf16((16, 512), 0.05, 9))
+    _compare(api.FMT_NVFP4, xb, noclip=True)
+    _compare(api.FMT_Q4_K, xb, noclip=True)
 
 
 def test_q4k_worked_and_degenerate():
