@@ -211,6 +211,29 @@ qf_status_t qf_pack(qf_layout_t layout, qf_format_t fmt, const void* codes, cons
 qf_status_t qf_unpack(qf_layout_t layout, qf_format_t fmt, const void* packed, int64_t rows, int64_t cols, void* codes,
                       void* scales, void* stream);
 
+/* The deployment-side product the fake-quantized layer stands for (Section 3.1, goal "Faithfulness to
+ * deployment"; Section 3.2: NVFP4 and MXFP4 are W4A4 formats at inference): Y = deq(A) . deq(B)^T computed by
+ * the block-scaled FP4 tensor-core instruction directly on the 4-bit codes and block scales that qf_qdq
+ * emitted for A [M,K] and B [N,K], FP32 accumulation, FP32 result. For MXFP4 this sums exactly the products
+ * the BF16 matmul of the training path sums (Eq. mxfp4-dequant is exact in BF16), so the two may differ only
+ * by FP32 summation order; for NVFP4 the training path additionally rounds each dequantized value to BF16
+ * (Eq. nvfp4-dequant), the native product does not, and the tensor scales multiply the accumulated sum.
+ * It is a checking tool for that equivalence (one CTA per 128x128 tile, not pipelined), not a serving kernel.
+ *   fmt          QF_FMT_MXFP4 or QF_FMT_NVFP4 (both operands)
+ *   a_codes      device, [M, K/2] bytes;  a_scales device, [M, K/32] E8M0 or [M, K/16] E4M3 bytes (row-major,
+ *                as qf_qdq writes them);  likewise b_codes / b_scales with N rows. Codes 16-byte aligned.
+ *   a_tscale, b_tscale  NVFP4: device float*, the tensor scales; ignored for MXFP4
+ *   Y            device float [M, N], 16-byte aligned
+ *   flags        QF_SCALES_TILED: a_scales and b_scales are in the tiled engine layout that qf_pack writes for
+ *                QF_LAYOUT_FP4_SWIZZLED_SCALES (16-byte aligned) instead of row-major: the 512-byte tiles are
+ *                handed to the tensor cores as they are, which is the hardware's own check of that layout
+ *   K % 32 == 0. workspace: at least qf_workspace_bytes(QF_OP_QDQ, ...) bytes; its status word reports an
+ *   expired device-side wait (qf_read_status). Errors as for the other calls. */
+#define QF_SCALES_TILED 0x100u
+qf_status_t qf_fp4_matmul_native(qf_format_t fmt, const void* a_codes, const void* a_scales, const float* a_tscale,
+                                 const void* b_codes, const void* b_scales, const float* b_tscale, int64_t M, int64_t N,
+                                 int64_t K, float* Y, uint32_t flags, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Allocation-free forward of the quantization-aware linear layer. (The paper has no counterpart:
  * this is a packaging variant of qf_fq_linear_fwd for hosts that cannot hand the library a workspace.)
  *

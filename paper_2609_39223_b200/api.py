@@ -19,6 +19,7 @@ TENSOR_SCALE_GIVEN = 0x1
 W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x2, 0x4, 0x8, 0x10
 REUSE_W_HAT, REUSE_X_HAT = 0x20, 0x40
 MXFP4_NO_CLIP = 0x80
+SCALES_TILED = 0x100
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 
@@ -28,6 +29,7 @@ EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
     "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack", "qf_nvfp4_tensor_scale", "qf_qdq_lora",
+    "qf_fp4_matmul_native",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 LAYOUT_GGUF_Q4_K, LAYOUT_FP4_SWIZZLED_SCALES = 1, 2
@@ -93,6 +95,9 @@ def lib() -> ctypes.CDLL:
         L.qf_pack.argtypes = [c_int, c_int, c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
         L.qf_unpack.restype = c_int
         L.qf_unpack.argtypes = [c_int, c_int, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
+        L.qf_fp4_matmul_native.restype = c_int
+        L.qf_fp4_matmul_native.argtypes = [c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64,
+                                           c_int64, c_void_p, c_uint32, c_void_p, c_size_t, c_void_p]
         L.qf_selftest_timeout.restype = c_int
         L.qf_selftest_timeout.argtypes = [c_void_p, c_size_t, c_int64, c_void_p]
         L.qf_selftest_mxfp4_bf16.restype = c_int
@@ -358,3 +363,18 @@ def qf_qdq_lora(fmt: int, W: torch.Tensor, B: torch.Tensor, A: torch.Tensor, lor
     _check(lib().qf_qdq_lora(fmt, _ptr(W), _ptr(B), _ptr(A), rank, float(lora_scale), rows, cols, _ptr(out), _ptr(codes),
                              _ptr(scales), _ptr(ts), flags, _ptr(ws), ws.numel(), _stream()), "qf_qdq_lora")
     return {"out": out, "codes": codes, "scales": scales, "tensor_scale": ts}
+
+
+def qf_fp4_matmul_native(fmt: int, a: dict, b: dict, K: int, *, flags: int = 0, ws=None) -> torch.Tensor:
+    """Y = deq(A) . deq(B)^T on the block-scaled FP4 tensor cores, from the dicts qf_qdq returned for
+    A [M, K] and B [N, K] (codes, scales and, for NVFP4, tensor_scale). Returns float32 [M, N].
+    With SCALES_TILED in ``flags`` the two ``scales`` entries are qf_pack's tiled block scales."""
+    M, N = a["codes"].shape[0], b["codes"].shape[0]
+    dev = a["codes"].device
+    Y = torch.empty((M, N), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(OP_QDQ, M, 0, K, device=dev)
+    _check(lib().qf_fp4_matmul_native(fmt, _ptr(a["codes"]), _ptr(a["scales"]), _ptr(a.get("tensor_scale")), _ptr(b["codes"]),
+                                      _ptr(b["scales"]), _ptr(b.get("tensor_scale")), M, N, K, _ptr(Y), flags, _ptr(ws), ws.numel(),
+                                      _stream()), "qf_fp4_matmul_native")
+    return Y

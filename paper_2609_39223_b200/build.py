@@ -13,7 +13,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libqf.so"
-SOURCES = ["qf_api.cu", "qf_qdq.cu", "qf_gemm.cu", "qf_pack.cu"]
+SOURCES = ["qf_api.cu", "qf_qdq.cu", "qf_gemm.cu", "qf_pack.cu", "qf_fp4_gemm.cu"]
 NVCC_FLAGS = [*os.environ.get("QF_EXTRA_NVCC", "").split(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -520,6 +520,34 @@ qf_status_t qf_unpack(qf_layout_t layout, qf_format_t fmt, const void* packed, i
   return cu(launch_swizzle_scales(packed, rows, cols / block_of(fmt), scales, true, st));
 }
 
+qf_status_t qf_fp4_matmul_native(qf_format_t fmt, const void* a_codes, const void* a_scales, const float* a_tscale,
+                                 const void* b_codes, const void* b_scales, const float* b_tscale, int64_t M, int64_t N,
+                                 int64_t K, float* Y, uint32_t flags, void* workspace, size_t workspace_bytes, void* stream) {
+  if (fmt != QF_FMT_MXFP4 && fmt != QF_FMT_NVFP4) return QF_ERR_FORMAT;
+  if (M < 0 || N < 0 || K < 0 || K % 32) return QF_ERR_SHAPE;
+  if (M > INT32_MAX - 128 || N > INT32_MAX - 128) return QF_ERR_SHAPE;             // tile coordinates are 32-bit
+  if (!workspace || workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;
+  if (M == 0 || N == 0) return QF_OK;
+  if (!Y) return QF_ERR_NULL;
+  if (K > 0 && (!a_codes || !a_scales || !b_codes || !b_scales)) return QF_ERR_NULL;
+  if (fmt == QF_FMT_NVFP4 && K > 0 && (!a_tscale || !b_tscale)) return QF_ERR_NULL;
+  if (!aligned16(a_codes) || !aligned16(b_codes) || !aligned16(Y) || !aligned16(workspace)) return QF_ERR_ALIGN;
+  if ((flags & QF_SCALES_TILED) && (!aligned16(a_scales) || !aligned16(b_scales))) return QF_ERR_ALIGN;
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* header = static_cast<uint32_t*>(workspace);
+  if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
+  Fp4GemmArgs g{};
+  g.scales_tiled = (flags & QF_SCALES_TILED) != 0;
+  g.fmt = fmt;
+  g.a_codes = a_codes; g.a_scales = a_scales; g.a_tscale = a_tscale;
+  g.b_codes = b_codes; g.b_scales = b_scales; g.b_tscale = b_tscale;
+  g.Y = Y;
+  g.M = M; g.N = N; g.K = K;
+  g.status_word = header + kWsStatus;
+  return cu(launch_fp4_native(g, st));
+}
+
 qf_status_t qf_selftest_timeout(void* workspace, size_t workspace_bytes, int64_t limit_cycles, void* stream) {
   if (!workspace) return QF_ERR_WORKSPACE;
   if (workspace_bytes < kWsHeader) return QF_ERR_WORKSPACE;

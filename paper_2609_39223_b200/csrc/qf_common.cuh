@@ -178,6 +178,22 @@ cudaError_t launch_pack_q4k(const void* codes, const void* scales, int64_t nsb, 
                             void* scales_out, cudaStream_t st);
 cudaError_t launch_swizzle_scales(const void* scales, int64_t rows, int64_t nblk, void* out, bool unswizzle, cudaStream_t st);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+
+// Operands of the native block-scaled FP4 product (qf_fp4_gemm.cu): codes and block scales as the quantizer emits them.
+struct Fp4GemmArgs {
+  int fmt;                           // QF_FMT_MXFP4 or QF_FMT_NVFP4
+  const void* a_codes;               // [M, K/2] bytes
+  const void* a_scales;              // [M, K/block] bytes
+  const void* b_codes;               // [N, K/2]
+  const void* b_scales;              // [N, K/block]
+  const float* a_tscale;             // NVFP4: device tensor scales
+  const float* b_tscale;
+  float* Y;                          // [M, N] FP32
+  int64_t M, N, K;
+  bool scales_tiled;                 // scales in the tiled engine layout (qf_pack, QF_LAYOUT_FP4_SWIZZLED_SCALES)
+  uint32_t* status_word;
+};
+cudaError_t launch_fp4_native(const Fp4GemmArgs& a, cudaStream_t st);
 bool gemm_can_fuse(const GemmArgs& a);
 cudaError_t launch_selftest_timeout(uint32_t* status, long long limit_cycles, int* gave_up, cudaStream_t st);
 
