@@ -14,7 +14,6 @@ namespace {
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ uint4 ld_chunk(const uint4* p) { return __ldg(p); }
 
 // Where a kernel's 16-byte input chunks come from. PlainLoader reads the tensor. LoraLoader produces
 // the chunk of the merged weight W + s * B A (Eq. qad-lora) on the fly, so the merged tensor is never
