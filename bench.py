@@ -302,14 +302,19 @@ def run_ours(args):
         out = torch.empty_like(Wq)
         codes = torch.empty((Wq.shape[0], Wq.shape[1] // 2), dtype=torch.uint8, device=dev)
         wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
-        for name, f in (("nvfp4", api.FMT_NVFP4), ("mxfp4", api.FMT_MXFP4), ("q4_k", api.FMT_Q4_K)):
+        given = torch.full((1,), 1e-4, dtype=torch.float32, device=dev)
+        # "nvfp4" derives the tensor scale from the tensor (an extra read of the whole input: the two passes move
+        # 6.56 B per element for 4.56 algorithmic, a ceiling of 0.70); "nvfp4_given_scale" is the mode with a
+        # tracked / tied tensor scale (QF_TENSOR_SCALE_GIVEN), one pass.
+        for name, f, ts in (("nvfp4", api.FMT_NVFP4, None), ("nvfp4_given_scale", api.FMT_NVFP4, given),
+                            ("mxfp4", api.FMT_MXFP4, None), ("q4_k", api.FMT_Q4_K, None)):
             sc = torch.empty(api.scales_shape(f, *Wq.shape), dtype=torch.uint8, device=dev)
             for _ in range(3):
-                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq)
+                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq, tensor_scale=ts)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for _ in range(10):
-                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq)
+                api.qf_qdq(f, Wq, out=out, codes=codes, scales=sc, ws=wsq, tensor_scale=ts)
             b.record(); torch.cuda.synchronize()
             bytes_per_elem = 2 + 2 + 0.5 + (1 / 32 if f == api.FMT_MXFP4 else 1 / 16)
             gbs = Wq.numel() * bytes_per_elem / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
