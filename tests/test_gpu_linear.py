@@ -122,6 +122,33 @@ def test_full_size_mxfp4_linear_sampled_rows():
     _close(dw[n_idx], oracle.matmul_wgrad(dyb, x_hat, n_idx), "dW rows")
 
 
+@pytest.mark.parametrize("y_dtype", [torch.float32, torch.bfloat16])
+def test_output_with_more_than_2_to_the_31_elements(y_dtype):
+    """A tall product whose output has 2.4e9 elements (and, in FP32, byte offsets past 2^33): sampled rows
+    around the 2^31-element boundary and at both ends against the oracle, forward and dX."""
+    M, N, K = 1048576, 2304, 64
+    assert M * N > 2 ** 31
+    X = synth.randn_bf16((M, K), 1.0, 31, device="cuda")
+    W = synth.randn_bf16((N, K), 0.05, 32, device="cuda")
+    fmt = api.FMT_MXFP4
+    y = api.qf_fq_linear_fwd(X, W, fmt, fmt, y_dtype=y_dtype)
+    boundary = 2 ** 31 // N
+    rows = [0, 1, 255, 256, boundary - 1, boundary, boundary + 1, M - 257, M - 2, M - 1]
+    xb, wb = torch_to_bits(X[rows].cpu()), torch_to_bits(W.cpu())
+    ref = oracle.fq_linear_fwd(xb, wb, fmt, fmt)
+    if y_dtype == torch.float32:
+        _close(y[rows], ref, "Y rows")
+    else:
+        _bf16_is_rounding_of(y[rows], torch.from_numpy(ref), "Y rows (BF16)")
+    assert bool((y != 0).any(dim=1).all())                       # no row was left unwritten
+    del y
+    # dX = dY . W_hat with the roles swapped: dY [M, N] is the large operand this time
+    dY = synth.randn_bf16((M, N), 1e-3, 33, device="cuda")
+    dx, _ = api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, dx_dtype=torch.float32, want_dw=False)
+    w_hat = oracle.qdq_out(fmt, wb)
+    _close(dx[rows], oracle.matmul_dgrad(torch_to_bits(dY[rows].cpu()), w_hat), "dX rows")
+
+
 def _grouped_reference(Xp, W, offs, wq, aq, dYp=None):
     G = W.shape[0]
     ys, dxs, dws = [], [], []

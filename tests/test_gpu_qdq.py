@@ -203,6 +203,34 @@ def test_full_size_mxfp4_activation():
     _compare(api.FMT_MXFP4, torch_to_bits(x))
 
 
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_more_than_2_to_the_31_elements(fmt, name):
+    """A tensor whose element count does not fit in 32 bits (36864 x 65536 = 2.4e9): every index in the
+    kernels must be 64-bit. Rows are independent given the tensor scale, so sampled rows from the start,
+    the middle, the 2^31-element boundary and the end are compared with the oracle run on those rows alone."""
+    rows, cols = 36864, 65536
+    assert rows * cols > 2 ** 31
+    x = synth.randn_bf16((rows, cols), 0.02, 17, device="cuda")
+    x[rows - 1, cols - 1] = 3.0                                  # the tensor maximum sits in the very last element
+    g = api.qf_qdq(fmt, x)
+    torch.cuda.synchronize()
+    ts = None
+    if fmt == api.FMT_NVFP4:
+        ts = float(g["tensor_scale"].item())
+        assert np.float32(ts) == np.float32(3.0) / np.float32(2688.0)
+    boundary = 2 ** 31 // cols
+    sample = [0, 1, rows // 3, boundary - 1, boundary, boundary + 1, rows - 2, rows - 1]
+    xb = torch_to_bits(x[sample].cpu())
+    o = oracle.qdq(fmt, xb, ts)
+    np.testing.assert_array_equal(torch_to_bits(g["out"][sample].cpu()), o["out"])
+    np.testing.assert_array_equal(g["codes"][sample].cpu().numpy(), o["codes"])
+    np.testing.assert_array_equal(g["scales"][sample].cpu().numpy(), o["scales"])
+    # nothing was left unwritten anywhere: the dequantized tensor is within one grid step of the input in every row
+    err = (g["out"].float() - x.float()).abs_().amax(dim=1)
+    assert float(err.max()) <= 0.5 and float(err.min()) > 0
+    del g, x
+
+
 def _guarded(nbytes, dtype, shape):
     """A tensor carved out of the middle of a larger byte buffer whose margins are filled with a canary."""
     pad = 1 << 16
