@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
 // ---------------------------------------------------------------------------------------------
 
 #ifndef QF_Q4K_MINBLOCKS
-#define QF_Q4K_MINBLOCKS 5      // 48 registers: five resident blocks per SM measured 4% faster than four
+#define QF_Q4K_MINBLOCKS 4      // 64 registers, no spills; five blocks (48 registers) measured the same within 1%
 #endif
 constexpr float kRcp15 = 1.0f / 15.0f;        // correctly rounded reciprocals of the two constant divisors
 constexpr float kRcp63 = 1.0f / 63.0f;
@@ -325,8 +325,9 @@ template <bool FAST>
 __device__ __forceinline__ float div_by(float x, float y, float rc) { return FAST ? div1_fast(x, y, rc) : __fdiv_rn(x, y); }
 
 template <bool FAST>
-__device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, float hi, uint32_t (&xhat)[16],
+__device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, float hi, uint4* __restrict__ out_ptr,
                                              uint32_t (&cbytes)[8], __half& d_h, __half& dmin_h, uint32_t& s6, uint32_t& m6) {
+  uint32_t xhat[4];
   lo = fminf(lo, 0.0f);
   const float sc = div_by<FAST>(__fsub_rn(hi, lo), 15.0f, kRcp15);
   const float off = __fsub_rn(0.0f, lo);            // >= +0: a sub-block with no negative value has offset +0
@@ -353,7 +354,7 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
   for (int j = 0; j < 16; ++j) {
     const float2 x = unpack2(w[j]);
     float2 y = magic;                                // code 0 when the sub-block has no scale
-    if (live) {
+    if (FAST || live) {                              // FAST: rc = 0 makes the reciprocal-based quotient 0, no branch needed
       const float2 num = __fadd2_rn(x, em2);
       float2 t = FAST ? div2_fast(num, es, rc) : make_float2(__fdiv_rn(num.x, es), __fdiv_rn(num.y, es));
       t.x = fminf(fmaxf(t.x, 0.0f), 15.0f);          // clamp first: rounding is monotone and 0, 15 are integers
@@ -362,7 +363,8 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
     }
     const float2 c = __fadd2_rn(y, nmagic);
     const float2 o = __ffma2_rn(es2, c, nem2);        // product exact: one rounding, as es*c - em
-    xhat[j] = pack_bf16x2(o.x, o.y);
+    xhat[j & 3] = pack_bf16x2(o.x, o.y);
+    if ((j & 3) == 3 && out_ptr) out_ptr[j >> 2] = make_uint4(xhat[0], xhat[1], xhat[2], xhat[3]);   // stored as soon as complete
     // the low byte of y's bit pattern is the code (the low byte of the rounding constant is zero)
     ybits[j & 1][0] = __float_as_uint(y.x);
     ybits[j & 1][1] = __float_as_uint(y.y);
@@ -402,14 +404,11 @@ __global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(Loa
     // tiny but non-zero range or offset takes the IEEE divide instead
     const float range = __fsub_rn(hi, fminf(lo, 0.0f)), offv = -fminf(lo, 0.0f);
     const bool fast_ok = (range == 0.0f || (range >= 0x1p-60f && range <= 0x1p60f)) && (offv == 0.0f || (offv >= 0x1p-60f && offv <= 0x1p60f));
-    uint32_t xhat[16], cb[8], s6, m6;
+    uint32_t cb[8], s6, m6;
     __half d_h, dmin_h;
-    if (__all_sync(0xFFFFFFFFu, fast_ok)) q4k_subblock<true>(w, lo, hi, xhat, cb, d_h, dmin_h, s6, m6);
-    else q4k_subblock<false>(w, lo, hi, xhat, cb, d_h, dmin_h, s6, m6);
-    if (ok && out) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) out[4 * i + k] = make_uint4(xhat[4 * k], xhat[4 * k + 1], xhat[4 * k + 2], xhat[4 * k + 3]);
-    }
+    uint4* const out_ptr = (ok && out) ? out + 4 * i : nullptr;
+    if (__all_sync(0xFFFFFFFFu, fast_ok)) q4k_subblock<true>(w, lo, hi, out_ptr, cb, d_h, dmin_h, s6, m6);
+    else q4k_subblock<false>(w, lo, hi, out_ptr, cb, d_h, dmin_h, s6, m6);
     // code bytes: a 64-element chunk is the lane pair (2j, 2j+1); byte l = code[2j][l] | code[2j+1][l] << 4.
     // cb[k] holds codes 4k..4k+3 one per byte. The even lane forms bytes 0-15, the odd lane bytes 16-31.
     const bool odd = lane & 1;
