@@ -106,6 +106,11 @@ __global__ void amax_to_scale_kernel(const uint32_t* amax_bits, float* scale) {
 // below keeps operands where that holds and the caller falls back to the IEEE divide otherwise.
 // qf_selftest_div compares it with the IEEE divide (tens of billions of pairs, including every BF16
 // numerator and divisors with an all-ones significand, without a difference).
+//
+// The residual is formed rounding toward minus infinity. Being exact, its value does not depend on the
+// rounding mode, but its sign when it is zero does: an exactly cancelling sum is -0 in that mode, so the
+// correction step adds -0 to q0 and leaves q0's sign alone. That makes x = -0 come out as -0, like the
+// IEEE quotient (with round-to-nearest the residual would be +0 and (+0) + (-0) = +0).
 // ---------------------------------------------------------------------------------------------
 
 #ifndef QF_DIV_STEPS
@@ -116,26 +121,23 @@ __global__ void amax_to_scale_kernel(const uint32_t* amax_bits, float* scale) {
 __device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
   const float2 ny = splat(-y), r = splat(rc);
   float2 q = __fmul2_rn(x, r);
-  q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
 #if QF_DIV_STEPS > 1
-  q = __ffma2_rn(__ffma2_rn(ny, q, x), r, q);
+  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
 #endif
   return q;
 }
 __device__ __forceinline__ float div1_fast(float x, float y, float rc) {
   float q = __fmul_rn(x, rc);
-  q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
 #if QF_DIV_STEPS > 1
-  q = __fmaf_rn(__fmaf_rn(-y, q, x), rc, q);
+  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
 #endif
   return q;
 }
 // divisor magnitudes for which the iteration above is used
 __device__ __forceinline__ bool div_safe(float y) { return y >= 0x1p-60f && y <= 0x1p60f; }
 
-__device__ __forceinline__ float copysign_bits(float mag, float sgn) {
-  return __uint_as_float((__float_as_uint(mag) & 0x7FFFFFFFu) | (__float_as_uint(sgn) & 0x80000000u));
-}
 
 
 
@@ -202,9 +204,7 @@ __device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const float2 x = unpack2(w[j]);
-      float2 v = div2_fast(x, S, rc);
-      v.x = copysign_bits(v.x, x.x);      // x = -0 must keep its sign, as in the IEEE quotient
-      v.y = copysign_bits(v.y, x.y);
+      const float2 v = div2_fast(x, S, rc);          // signed zeros included: x = -0 gives -0
       const uint32_t byte = e2m1x2_encode(v.x, v.y);
       const float2 o = __fmul2_rn(__fmul2_rn(sb2, e2m1x2_decode(byte)), st2);
       r.xhat[j] = pack_bf16x2(o.x, o.y);
@@ -470,9 +470,9 @@ __global__ void selftest_div_kernel(const float* __restrict__ xs, int64_t nx, co
     if (!(x == 0.0f || fabsf(x) >= 0x1p-60f || fabsf(ref) >= 0x1p-8f) || fabsf(ref) > 0x1p100f) continue;
     const float2 q = div2_fast(make_float2(x, -x), y, rc);
     const float q1 = div1_fast(x, y, rc);
-    if (__float_as_uint(copysign_bits(q.x, x)) != __float_as_uint(ref)) ++bad;
-    if (__float_as_uint(copysign_bits(q.y, -x)) != __float_as_uint(-ref)) ++bad;
-    if (__float_as_uint(copysign_bits(q1, x)) != __float_as_uint(ref)) ++bad;
+    if (__float_as_uint(q.x) != __float_as_uint(ref)) ++bad;             // bit patterns: the sign of a zero counts
+    if (__float_as_uint(q.y) != __float_as_uint(-ref)) ++bad;
+    if (__float_as_uint(q1) != __float_as_uint(ref)) ++bad;
   }
   if (bad) atomicAdd(mismatches, bad);
 }
