@@ -231,10 +231,13 @@ def test_full_size_nvfp4_weight_only_32k_tokens_sampled_rows():
     _close(dw[torch.from_numpy(n_idx).cuda()], dw_ref, "dW rows")
 
 
-def test_full_size_moe_grouped_mxfp4_sampled_experts():
-    """128 experts, hidden 2048, expert MLP 768, 16384 tokens routed top-8: the gate/up projection
-    (N=768, K=2048) forward and backward over all 131072 routed rows; three experts checked in full."""
-    tokens, E, top_k, H, F = 16384, 128, 8, 2048, 768
+@pytest.mark.parametrize("shape", ["gate", "gate_up", "down"])
+def test_full_size_moe_grouped_mxfp4_sampled_experts(shape):
+    """128 experts, hidden 2048, expert MLP 768, 16384 tokens routed top-8: the gate projection
+    (N=768, K=2048), gate and up as one weight (N=1536, the layout the benchmark times) and the down
+    projection (N=2048, K=768), forward and backward over all 131072 routed rows; three experts checked in full."""
+    tokens, E, top_k = 16384, 128, 8
+    F, H = {"gate": (768, 2048), "gate_up": (1536, 2048), "down": (2048, 768)}[shape]      # F = N, H = K of this projection
     r = synth.moe_routing(tokens, E, top_k, seed=0)
     assert abs(int(r.counts.sum()) - tokens * top_k) == 0 and int(r.counts.min()) > 0
     X = synth.randn_bf16((tokens, H), 1.0, 1)
