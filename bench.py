@@ -323,7 +323,7 @@ def run_ours(args):
             bytes_per_elem = 2 + 2 + 0.5 + (1 / 32 if f == api.FMT_MXFP4 else 1 / 16)
             gbs = Wq.numel() * bytes_per_elem / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
             qdq[name] = {"gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
-                         "bytes_per_elem": bytes_per_elem}
+                         "frac_of_8000_nominal": round(gbs / 8000.0, 4), "bytes_per_elem": bytes_per_elem}
         del Wq, out, codes
 
     # ---- headline: K steps, inputs resident in HBM -------------------------------------------------
