@@ -75,6 +75,7 @@ inline float e2m1_value(uint8_t code) {
 // The sign bit is copied from v even when the magnitude rounds to zero.
 inline uint8_t e2m1_encode(float v) {
     double a = std::fabs(static_cast<double>(v));
+    if (a > 6.0) a = 6.0;      // saturate first: for huge |v| every distance |a - grid| rounds to the same double
     int best = 0;
     double best_d = std::fabs(a - kE2M1Mag[0]);
     for (int c = 1; c < 8; ++c) {

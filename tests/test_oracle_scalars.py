@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import oracle
+from util import bits_to_f32, f32_to_bits
 
 GOLDEN = Path(__file__).parent / "golden"
 
@@ -46,6 +47,17 @@ def test_e2m1_one_ulp_around_every_midpoint():
         assert oracle.e2m1_value(oracle.e2m1_encode(below)) == lo
         assert oracle.e2m1_value(oracle.e2m1_encode(above)) == hi
         assert oracle.e2m1_encode(mid) % 2 == 0                 # the tie goes to the even code
+
+
+def test_e2m1_saturates_at_6_however_large_the_value():
+    # Eq. e2m1-values: 6 is the largest magnitude of the grid, so everything beyond it lands there, including
+    # values so large that their distances to all grid points coincide in double precision
+    for v in (6.0, 6.5, 8.0, 1e9, 2.0 ** 53, 2.0 ** 54 + 2.0 ** 31, 1e20, 3.7e25, 3.0e38, float(np.finfo(np.float32).max)):
+        assert oracle.e2m1_encode(v) == 7 and oracle.e2m1_encode(-v) == 15, v
+    x = np.zeros((1, 32), np.float32); x[0, 0] = 1.6557448e28; x[0, 1] = -1.0154977e27; x[0, 2] = 448 * 5.5
+    r = oracle.qdq(oracle.FMT_NVFP4, f32_to_bits(x), 1.0)          # a supplied tensor scale far too small: block scale 448
+    assert r["scales"][0, 0] == 0x7E
+    assert list(bits_to_f32(r["out"])[0, :3]) == [2688.0, -2688.0, 2688.0]
 
 
 def test_e2m1_matches_ml_dtypes_cast():
