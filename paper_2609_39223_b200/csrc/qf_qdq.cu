@@ -187,7 +187,11 @@ __device__ __forceinline__ UnitOut mxfp4_unit(const uint32_t (&w)[8], uint32_t b
 template <bool FAST>
 __device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax_b, float s_t, float denom, float rc_denom,
                                               uint32_t& scale_code) {
-  const float q = FAST ? div1_fast(amax_b, denom, rc_denom) : __fdiv_rn(amax_b, denom);
+  // A supplied tensor scale can be far too small for a block: the quotient then exceeds every E4M3 value and may
+  // even overflow FP32, which the reciprocal-based form does not survive (inf - inf). 512 * denom is exact
+  // (denom lies in [2^-60, 2^60] on this path); at or beyond it the scale is the largest code whatever the quotient.
+  const float q = FAST ? (amax_b >= __fmul_rn(512.0f, denom) ? 512.0f : div1_fast(amax_b, denom, rc_denom))
+                       : __fdiv_rn(amax_b, denom);
   scale_code = e4m3_encode(q);
   const float sb = e4m3_decode(scale_code);
   const float S = __fmul_rn(s_t, sb);
