@@ -79,16 +79,16 @@ def test_wide_dynamic_range_blocks(fmt, name):
     _compare(fmt, f32_to_bits(x))
 
 
-def _random_bit_patterns(rng, rows, cols, group):
+def _random_bit_patterns(rng, rows, cols, group, top=220):
     """Raw BF16 bit patterns: every `group` elements share an exponent centre drawn from the whole range in use
     (biased exponent 0 = subnormals up to 220 = 2^93; beyond that differences of two values can overflow FP32,
     which the formats' arithmetic is not defined for), individual exponents scatter around it by a per-group
     spread of 0 to 40 binades, mantissas and signs are uniform, and a tenth of the groups get zeros mixed in."""
     ng = rows * cols // group
-    centre = rng.integers(0, 221, ng)
+    centre = rng.integers(0, top + 1, ng)
     spread = rng.choice([0, 1, 3, 8, 20, 40], ng)
     e = centre[:, None] + np.rint(rng.normal(0, 1, (ng, group)) * spread[:, None]).astype(np.int64)
-    e = np.clip(e, 0, 220)
+    e = np.clip(e, 0, top)
     bits = (rng.integers(0, 2, (ng, group)) << 15) | (e << 7) | rng.integers(0, 128, (ng, group))
     zero = (rng.random((ng, 1)) < 0.1) & (rng.random((ng, group)) < 0.5)
     bits[zero] &= 0x8000                                   # +0 and -0
@@ -105,6 +105,11 @@ def test_random_bit_patterns_over_the_whole_exponent_range(fmt, name, seed):
     if fmt == api.FMT_NVFP4:
         for ts in (2.0 ** -40, 3.7e-9, 1.0, 2.0 ** 20):
             _compare(fmt, x, tensor_scale=ts)
+    if fmt == api.FMT_MXFP4:
+        _compare(fmt, x, noclip=True)
+    if fmt != api.FMT_Q4_K:
+        # the two FP4 formats never subtract two inputs, so every finite BF16 value is fair game
+        _compare(fmt, _random_bit_patterns(rng, 64, 4096, group, top=254))
 
 
 def test_nvfp4_exact_ties_and_given_scale():
