@@ -302,6 +302,36 @@ def test_mxfp4_scale_rule_without_saturation_through_the_layer(wq, aq, M, N, K):
     assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
 
 
+def test_in_kernel_quantization_on_blocks_at_the_bottom_of_the_exponent_range():
+    """The in-kernel transform rounds in packed BF16 arithmetic for ordinary blocks and falls back to the
+    conversion route for all-zero blocks and blocks whose scale sits at either end of the exponent range.
+    Operands that mix ordinary blocks with zero, subnormal and tiny ones must still give the default path's
+    bits (compared as bit patterns), and finite results."""
+    M, N, K = 512, 512, 1024
+    rng = np.random.default_rng(77)
+    def operand(rows):
+        ng = rows * K // 32
+        kind = rng.integers(0, 4, ng)                                   # 0 ordinary, 1 zero, 2 subnormal, 3 tiny normal
+        e = np.where(kind == 0, rng.integers(110, 135, ng), np.where(kind == 2, 0, rng.integers(1, 12, ng)))
+        bits = (rng.integers(0, 2, (ng, 32)) << 15) | ((e[:, None] + rng.integers(0, 3, (ng, 32))) << 7) | rng.integers(0, 128, (ng, 32))
+        bits[kind == 1] &= 0x8000
+        bits[kind == 2] &= 0x807F
+        return torch.from_numpy(bits.astype(np.uint16).reshape(rows, K).view(np.int16)).view(torch.bfloat16).cuda()
+    X, W = operand(M), operand(N)
+    dY = synth.randn_bf16((M, N), 1e-3, 5, device="cuda")
+    fmt = api.FMT_MXFP4
+    y0 = api.qf_fq_linear_fwd(X, W, fmt, fmt, y_dtype=torch.float32)
+    dx0, dw0 = api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32)
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    y1 = api.qf_fq_linear_fwd(X, W, fmt, fmt, y_dtype=torch.float32, flags=api.FUSED_QDQ, ws=ws)
+    dx1, dw1 = api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32, flags=api.FUSED_QDQ, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    for a, b in ((y0, y1), (dx0, dx1), (dw0, dw1)):
+        assert bool(torch.isfinite(a).all())
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    _close(y1, oracle.fq_linear_fwd(torch_to_bits(X.cpu()), torch_to_bits(W.cpu()), fmt, fmt), "Y")
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
     status word and leave the context usable (no trap, no hang)."""
