@@ -43,6 +43,28 @@ def test_oracle_quantizes_the_merged_weight_not_the_base():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("fmt", [api.FMT_NVFP4, api.FMT_MXFP4, api.FMT_Q4_K])
+def test_gpu_fused_merge_on_wide_range_bit_patterns(fmt):
+    """Base weight and factors drawn as raw BF16 bit patterns over forty binades, signs and zeros mixed in:
+    the merge's FP32 accumulation order and its single BF16 rounding must agree bit for bit whatever cancels."""
+    rng = np.random.default_rng(123)
+    rows, cols, rank = 96, 1024, 12
+    def pat(shape, lo, hi):
+        n = int(np.prod(shape))
+        bits = (rng.integers(0, 2, n) << 15) | (rng.integers(lo, hi, n) << 7) | rng.integers(0, 128, n)
+        bits[rng.random(n) < 0.05] &= 0x8000
+        return bits.astype(np.uint16).reshape(shape)
+    w, b, a = pat((rows, cols), 100, 140), pat((rows, rank), 110, 130), pat((rank, cols), 110, 130)
+    to_t = lambda x: torch.from_numpy(x.view(np.int16).copy()).view(torch.bfloat16).cuda()
+    for scale in (1.0, -0.37, 1024.0):
+        g = api.qf_qdq_lora(fmt, to_t(w), to_t(b), to_t(a), scale)
+        o = oracle.qdq_lora(fmt, w, b, a, scale)
+        np.testing.assert_array_equal(torch_to_bits(g["out"]), o["out"])
+        np.testing.assert_array_equal(g["codes"].cpu().numpy(), o["codes"])
+        np.testing.assert_array_equal(g["scales"].cpu().numpy(), o["scales"])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("fmt", [api.FMT_NVFP4, api.FMT_MXFP4, api.FMT_Q4_K])
 @pytest.mark.parametrize("rows,cols,rank,scale", [(1, 256, 1, 1.0), (37, 768, 16, 2.0), (300, 1024, 64, 0.5), (64, 512, 0, 1.0)])
 def test_gpu_fused_merge_and_quantize_is_bit_exact(fmt, rows, cols, rank, scale):
     w, b, a = _case(rows, cols, max(rank, 1), rows + rank)
