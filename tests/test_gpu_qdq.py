@@ -112,6 +112,27 @@ def test_random_bit_patterns_over_the_whole_exponent_range(fmt, name, seed):
         _compare(fmt, _random_bit_patterns(rng, 64, 4096, group, top=254))
 
 
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_dequantizer_alone_on_arbitrary_codes_and_metadata(fmt, name):
+    """Q^-1 on its own (the path a checkpoint reader takes): every code byte, every valid scale byte, arbitrary
+    finite FP16 super-block factors and 6-bit fields, not only combinations the quantizer would emit."""
+    rng = np.random.default_rng(31)
+    rows, cols = 64, 2048
+    codes = rng.integers(0, 256, (rows, cols // 2), dtype=np.uint8)
+    if fmt == api.FMT_NVFP4:
+        scales = rng.integers(0, 0x7F, (rows, cols // 16), dtype=np.uint8)           # E4M3 codes 0x00..0x7E
+    elif fmt == api.FMT_MXFP4:
+        scales = rng.integers(0, 255, (rows, cols // 32), dtype=np.uint8)            # E8M0 codes 0..254
+    else:
+        scales = rng.integers(0, 256, (rows, cols // 256, 16), dtype=np.uint8)
+        half = rng.integers(0, 0x7C00, (rows, cols // 256, 2)).astype(np.uint16)     # finite non-negative FP16 d, dmin
+        scales[..., 0:4] = half.view(np.uint8).reshape(rows, cols // 256, 4)
+    for ts in ((3.1e-5, 1.0, 2.0 ** 30) if fmt == api.FMT_NVFP4 else (None,)):
+        t = None if ts is None else torch.tensor([ts], dtype=torch.float32, device="cuda")
+        d = api.qf_dequant(fmt, torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda(), t, rows, cols)
+        np.testing.assert_array_equal(torch_to_bits(d), oracle.dequant(fmt, codes, scales, ts, rows, cols))
+
+
 def test_nvfp4_exact_ties_and_given_scale():
     # with s_t = 2^-10 and a block maximum of 2.625 the block scale is 448 and S = 7/16, so these
     # inputs sit exactly on the rounding midpoints 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5 (times S)
