@@ -56,6 +56,33 @@ def test_small_complete_shapes(wq, aq, M, N, K):
     _bf16_is_rounding_of(dw16, dw32, "dW bf16")
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        M = int(rng.choice([rng.integers(1, 128), rng.integers(128, 300), rng.integers(300, 900)]))
+        N = 8 * int(rng.integers(1, 100))
+        K = 32 * int(rng.integers(1, 48))
+        out.append((M, N, K))
+    return out
+
+
+@pytest.mark.parametrize("M,N,K", _random_shapes(14, 2024))
+def test_randomly_drawn_shapes(M, N, K):
+    """Shapes drawn at random across the one-CTA / two-CTA dispatch boundary (256 rows), with ragged row, column
+    and contraction tails in every combination, forward and both backward products, with and without quantizers."""
+    c = synth.linear_case(M, N, K, seed=M * 7 + N + K, outlier_channels=1)
+    xb, wb, dyb = (torch_to_bits(t) for t in (c.X, c.W, c.dY))
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    for wq, aq in ((api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NONE, api.FMT_NONE), (api.FMT_NVFP4, api.FMT_NVFP4)):
+        y = api.qf_fq_linear_fwd(X, W, wq, aq, y_dtype=torch.float32)
+        dx, dw = api.qf_fq_linear_bwd(dY, X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32)
+        _close(y, oracle.fq_linear_fwd(xb, wb, wq, aq), f"Y {wq}/{aq}")
+        dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, wq, aq)
+        _close(dx, dx_ref, f"dX {wq}/{aq}")
+        _close(dw, dw_ref, f"dW {wq}/{aq}")
+
+
 def test_one_hot_rows_read_out_quantized_weights_exactly():
     K, N = 256, 264
     W = synth.randn_bf16((N, K), 0.02, 1).cuda()
