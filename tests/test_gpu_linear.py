@@ -214,6 +214,39 @@ def test_grouped_small_with_ragged_and_empty_experts(wq, aq):
     _close(dw, dw_ref, "grouped dW")
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_grouped_randomly_drawn_segments(seed):
+    """Expert counts, segment lengths (zero included; each padded to a multiple of 128 rows as the interface
+    requires), widths and contraction lengths drawn at random: both grouped kernels (the two-CTA one and the
+    one-CTA one it falls back to for short problems) against the per-expert oracle."""
+    rng = np.random.default_rng(500 + seed)
+    E = int(rng.integers(1, 12))
+    blocks = rng.choice([0, 1, 1, 2, 3, 5], E)                      # 128-row blocks per expert
+    if seed % 2 == 0:
+        blocks[:] = np.minimum(blocks, 1)                            # short problems: fewer than 256 rows in total sometimes
+    offs = torch.tensor(np.concatenate([[0], np.cumsum(blocks) * 128]), dtype=torch.int32)
+    rows = int(offs[-1])
+    if rows == 0:
+        blocks[0] = 1; offs = torch.tensor(np.concatenate([[0], np.cumsum(blocks) * 128]), dtype=torch.int32); rows = int(offs[-1])
+    F, H = 8 * int(rng.integers(1, 60)), 32 * int(rng.integers(1, 24))
+    Xp = synth.randn_bf16((rows, H), 1.0, 10 + seed)
+    real = torch.ones(rows, dtype=torch.bool)
+    for g in range(E):                                               # the tail of each segment is padding: zero rows
+        a, b = int(offs[g]), int(offs[g + 1])
+        if b > a:
+            real[b - int(rng.integers(0, 100)):b] = False
+    Xp[~real] = 0
+    W = synth.randn_bf16((E, F, H), 0.02, 20 + seed)
+    dYp = synth.randn_bf16((rows, F), 1e-3, 30 + seed); dYp[~real] = 0
+    for wq, aq in ((api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NONE, api.FMT_NONE)):
+        y_ref, dx_ref, dw_ref = _grouped_reference(Xp, W, offs, wq, aq, dYp)
+        y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), wq, aq, y_dtype=torch.float32)
+        dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32)
+        _close(y, y_ref, "grouped Y")
+        _close(dx, dx_ref, "grouped dX")
+        _close(dw, dw_ref, "grouped dW")
+
+
 def test_grouped_empty_expert_gives_zero_dw():
     E, H, F = 3, 256, 256
     offs = torch.tensor([0, 128, 128, 256], dtype=torch.int32)        # expert 1 has no rows
