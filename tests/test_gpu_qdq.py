@@ -133,6 +133,22 @@ def test_dequantizer_alone_on_arbitrary_codes_and_metadata(fmt, name):
         np.testing.assert_array_equal(torch_to_bits(d), oracle.dequant(fmt, codes, scales, ts, rows, cols))
 
 
+def test_amax_over_odd_lengths_and_negative_maxima():
+    """max|x| over tensors whose length is not a multiple of the 8-element load width, with the maximum placed in the
+    ragged tail, at the front, and carried by a negative value; and over several tensors at once."""
+    rng = np.random.default_rng(8)
+    for n in (1, 7, 8, 9, 1023, 4097, 70001, 1 << 20 | 5):
+        x = synth.randn_bf16((n,), 1.0, n, device="cuda")
+        for pos, val in ((n - 1, -37.5), (0, 41.0), (int(rng.integers(0, n)), -53.0)):
+            x[pos] = val
+            assert api.qf_amax(x).item() == abs(val)
+    parts = [synth.randn_bf16((m,), 1.0, 3 * m, device="cuda") for m in (5, 4096, 33, 100003)]
+    parts[2][17] = -99.0
+    state = torch.zeros(1, dtype=torch.float32, device="cuda")
+    scale = api.qf_nvfp4_tensor_scale(parts, state)
+    assert state.item() == 99.0 and np.float32(scale.item()) == np.float32(99.0) / np.float32(2688.0)
+
+
 def test_nvfp4_exact_ties_and_given_scale():
     # with s_t = 2^-10 and a block maximum of 2.625 the block scale is 448 and S = 7/16, so these
     # inputs sit exactly on the rounding midpoints 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5 (times S)
