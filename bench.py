@@ -241,7 +241,7 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
     r = synth.moe_routing(tokens, E, top_k, seed=0)
     rows = int(r.group_offsets[-1]); offs = r.group_offsets.to(dev)
     fmt = api.FMT_MXFP4
-    tot_ms = 0.0
+    tot_ms, tot_reuse_ms = 0.0, 0.0
     for (Nn, Kk, times) in ((2 * F, H, 1), (H, F, 1)):
         Xp = synth.randn_bf16((rows, Kk), 1.0, 5, device=dev); Xp[(r.token_of_row < 0).to(dev)] = 0
         Wg = synth.randn_bf16((E, Nn, Kk), 0.02, 6, device=dev)
@@ -253,11 +253,17 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
         def f5():
             api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
             api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dW)
+
+        def f5_reuse():          # the backward keeps the forward's fake-quantized copies instead of recomputing them
+            api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
+            api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dW, flags=api.REUSE_W_HAT | api.REUSE_X_HAT)
         tot_ms += times * _time_ms(torch, f5, reps=10, warm=3)
+        tot_reuse_ms += times * _time_ms(torch, f5_reuse, reps=10, warm=3)
         del Xp, Wg, dYp, ws5, Y, dX, dW
     fl = 3 * 3 * 2.0 * tokens * top_k * H * F
     out["moe_grouped_mxfp4_128_experts"] = {"ms": tot_ms, "tflops": fl / (tot_ms * 1e-3) / 1e12, "routed_rows": tokens * top_k,
                                             "layout": "gate and up as one [128, 1536, 2048] grouped weight, down [128, 2048, 768]",
+                                            "ms_reusing_forward_copies": tot_reuse_ms, "tflops_reusing_forward_copies": fl / (tot_reuse_ms * 1e-3) / 1e12,
                                             "padded_rows": rows, "frac_of_2250_datasheet": fl / (tot_ms * 1e-3) / 1e12 / 2250.0}
     return out
 
