@@ -94,6 +94,15 @@ __global__ void amax_to_scale_kernel(const uint32_t* amax_bits, float* scale) {
   *scale = a == 0.0f ? 1.0f : __fdiv_rn(a, 2688.0f);
 }
 
+// the same for an array of maxima, converted where they stand (one tensor scale per expert)
+__global__ void amax_to_scale_inplace_kernel(uint32_t* bits, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    const float a = __uint_as_float(bits[i]);
+    bits[i] = __float_as_uint(a == 0.0f ? 1.0f : __fdiv_rn(a, 2688.0f));
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Exact division without the per-element IEEE divide sequence.
 //
@@ -674,12 +683,18 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
   QdqArgs q = a;
   q.tscale_in = nullptr;
   if (a.groups > 1) {
-    // per-expert tensor scales: the caller's scale array doubles as the amax accumulator (FP32 bits of a
-    // non-negative value), which the quantize pass then overwrites with the derived scales
+    // per-expert tensor scales: the caller's scale array first accumulates the maxima (FP32 bits of a
+    // non-negative value) and is then converted to the derived scales
     uint32_t* bits = reinterpret_cast<uint32_t*>(a.tscale_out);
     if (cudaError_t e = cudaMemsetAsync(bits, 0, sizeof(uint32_t) * a.groups, st)) return e;
     if (cudaError_t e = launch_amax_grouped(a.in, a.rows * a.cols / a.groups, a.groups, bits, st)) return e;
-    q.amax_bits = bits;
+    // The maxima become scales in place before the quantize pass starts: that pass must find finished scales,
+    // not words that one of its own CTAs is still turning from a maximum into a scale.
+    amax_to_scale_inplace_kernel<<<(a.groups + kThreads - 1) / kThreads, kThreads, 0, st>>>(bits, a.groups);
+    if (cudaError_t e = cudaGetLastError()) return e;
+    q.tscale_in = a.tscale_out;
+    q.tscale_out = nullptr;
+    q.amax_bits = nullptr;
     return launch_qdq(q, st);
   }
   uint32_t* amax_bits = header + amax_word;
