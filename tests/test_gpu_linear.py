@@ -475,6 +475,23 @@ def test_grouped_nvfp4_weights_have_one_tensor_scale_per_expert():
         api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NONE)
 
 
+def test_grouped_nvfp4_scales_are_final_before_any_block_is_quantized():
+    """Experts large enough that many CTAs quantize each one: all of them must use the expert's finished tensor
+    scale. Repeated, because a CTA that converted the shared word too early would only sometimes be caught."""
+    E, H, F = 4, 1024, 1024
+    offs = torch.tensor([0, 128, 256, 384, 512], dtype=torch.int32)
+    Xp = torch.eye(128, H, dtype=torch.bfloat16).repeat(E, 1)                       # one-hot rows read out W_hat[:, :128]
+    W = synth.randn_bf16((E, F, H), 0.02, 21)
+    W = (W.float() * torch.tensor([1.0, 8.0, 0.125, 64.0]).view(E, 1, 1)).to(torch.bfloat16)
+    want = [bits_to_f32(oracle.qdq_out(api.FMT_NVFP4, torch_to_bits(W[g])))[:, :128].T for g in range(E)]
+    Xd, Wd, od = Xp.cuda(), W.cuda(), offs.cuda()
+    for _ in range(10):
+        wts = torch.zeros(E, device="cuda")
+        y = api.qf_fq_grouped_linear_fwd(Xd, Wd, od, api.FMT_NVFP4, api.FMT_NONE, y_dtype=torch.float32, w_tscale=wts).cpu().numpy()
+        for g in range(E):
+            np.testing.assert_array_equal(y[g * 128:(g + 1) * 128], want[g])
+
+
 @pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NVFP4, api.FMT_NVFP4), (api.FMT_Q4_K, api.FMT_NONE)])
 def test_backward_can_reuse_the_forwards_quantized_copies(wq, aq):
     M, N, K = 384, 520, 1024
