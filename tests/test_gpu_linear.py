@@ -392,6 +392,35 @@ def test_in_kernel_quantization_on_blocks_at_the_bottom_of_the_exponent_range():
     _close(y1, oracle.fq_linear_fwd(torch_to_bits(X.cpu()), torch_to_bits(W.cpu()), fmt, fmt), "Y")
 
 
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_NVFP4, api.FMT_NVFP4), (api.FMT_Q4_K, api.FMT_NONE)])
+def test_a_whole_step_replays_from_a_cuda_graph(wq, aq):
+    """Nothing in a call synchronises, allocates or reads device memory on the host, so forward and backward
+    can be captured into a CUDA graph; replays with new input contents must equal the eager results bit for bit."""
+    M, N, K = 512, 768, 1024
+    c = synth.linear_case(M, N, K, seed=9, outlier_channels=2)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda"); dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    wts, ats = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+
+    def step():
+        api.qf_fq_linear_fwd(X, W, wq, aq, ws=ws, Y=Y, w_tscale=wts, a_tscale=ats)
+        api.qf_fq_linear_bwd(dY, X, W, wq, aq, ws=ws, dX=dX, dW=dW, w_tscale=wts, a_tscale=ats)
+    step(); torch.cuda.synchronize()                       # first use outside capture (per-device kernel attributes)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for seed in (1, 2):
+        c2 = synth.linear_case(M, N, K, seed=100 + seed, outlier_channels=2)
+        X.copy_(c2.X); W.copy_(c2.W); dY.copy_(c2.dY)
+        g.replay(); torch.cuda.synchronize()
+        got = (Y.clone(), dX.clone(), dW.clone())
+        step(); torch.cuda.synchronize()
+        assert torch.equal(got[0], Y) and torch.equal(got[1], dX) and torch.equal(got[2], dW)
+        assert api.qf_read_status(ws) == 0
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
     status word and leave the context usable (no trap, no hang)."""
