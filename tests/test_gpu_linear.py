@@ -421,6 +421,34 @@ def test_a_whole_step_replays_from_a_cuda_graph(wq, aq):
         assert api.qf_read_status(ws) == 0
 
 
+def test_independent_calls_on_two_streams():
+    """Two layers, each with its own workspace, driven from two streams at once: the results are those of running
+    them one after the other (the library keeps no state between calls)."""
+    shapes = [(640, 512, 1024), (384, 1024, 512)]
+    cases = [synth.linear_case(M, N, K, seed=40 + i, outlier_channels=1, device="cuda") for i, (M, N, K) in enumerate(shapes)]
+    fmt = api.FMT_MXFP4
+    serial = []
+    for c, (M, N, K) in zip(cases, shapes):
+        y = api.qf_fq_linear_fwd(c.X, c.W, fmt, fmt, y_dtype=torch.float32)
+        dx, dw = api.qf_fq_linear_bwd(c.dY, c.X, c.W, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32)
+        serial.append((y, dx, dw))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    wss = [api.workspace(api.OP_LINEAR_BWD, *s) for s in shapes]
+    for rep in range(5):
+        outs = [None, None]
+        for i in (0, 1):
+            with torch.cuda.stream(streams[i]):
+                c = cases[i]
+                y = api.qf_fq_linear_fwd(c.X, c.W, fmt, fmt, y_dtype=torch.float32, ws=wss[i])
+                dx, dw = api.qf_fq_linear_bwd(c.dY, c.X, c.W, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=wss[i])
+                outs[i] = (y, dx, dw)
+        torch.cuda.synchronize()
+        for i in (0, 1):
+            assert all(torch.equal(a, b) for a, b in zip(outs[i], serial[i]))
+            assert api.qf_read_status(wss[i]) == 0
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
     status word and leave the context usable (no trap, no hang)."""
