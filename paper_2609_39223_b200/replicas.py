@@ -46,6 +46,17 @@ def aggregate_rate(units_per_rank: float, elapsed_ms_this_rank: float, device="c
     return n * units_per_rank / (ms * 1e-3), ms
 
 
+def allreduce_max_(t: torch.Tensor) -> torch.Tensor:
+    """In-place MAX over ranks of a small tensor. The one exchange a row-sharded NVFP4 weight needs: its tensor
+    scale is a property of the whole tensor, so every rank reduces the absolute maximum of its shard
+    (``qf_nvfp4_tensor_scale(..., want_scale=False)``), the 4-byte maxima are combined here, and the combined value
+    becomes the shared scale (``qf_nvfp4_tensor_scale([], state, running=True)``) that each rank then supplies to
+    ``qf_qdq`` / the linear calls. Blocks, rows and the other two formats need no exchange at all."""
+    if dist.is_initialized():
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t
+
+
 def finish() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

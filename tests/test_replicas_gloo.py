@@ -48,6 +48,52 @@ def test_two_gloo_ranks_agree_on_max_time_and_aggregate_rate(tmp_path):
         assert f"rank {rank} ok" in out
 
 
+SHARD_WORKER = textwrap.dedent("""
+    import sys
+    sys.path.insert(0, %r); sys.path.insert(0, %r)
+    import numpy as np, torch
+    import oracle
+    from paper_2609_39223_b200 import replicas, synth
+    from util import torch_to_bits
+    n, rank, local = replicas.world()
+    replicas.init("gloo")
+    W = synth.weight_with_outliers(64, 512, seed=3)              # the same full weight on both ranks (seeded)
+    W[40, 7] = 1.75                                              # the tensor maximum lives in rank 1's half
+    full = oracle.qdq(oracle.FMT_NVFP4, torch_to_bits(W))
+    shard = W[rank * 32:(rank + 1) * 32]
+    state = torch.tensor([float(shard.float().abs().max())], dtype=torch.float32)
+    replicas.allreduce_max_(state)
+    assert state.item() == 1.75
+    scale = np.float32(state.item()) / np.float32(2688.0)
+    assert scale == np.float32(full["tensor_scale"])
+    mine = oracle.qdq(oracle.FMT_NVFP4, torch_to_bits(shard), float(scale))
+    for k in ("out", "codes", "scales"):
+        np.testing.assert_array_equal(mine[k], full[k][rank * 32:(rank + 1) * 32])
+    if rank == 0:                                                # without the exchange rank 0 would pick a different scale
+        alone = oracle.qdq(oracle.FMT_NVFP4, torch_to_bits(shard))
+        assert np.float32(alone["tensor_scale"]) != scale
+    replicas.finish()
+    print("rank", rank, "ok")
+""" % (str(ROOT), str(ROOT / "tests")))
+
+
+def test_row_sharded_nvfp4_weight_shares_one_tensor_scale(tmp_path):
+    """A weight split by rows over two ranks: one 4-byte MAX all-reduce of the shard maxima gives every rank the
+    tensor scale of the whole weight, and each shard then quantizes to exactly its rows of the unsharded result."""
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER)
+    port = _free_port()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, WORLD_SIZE="2", RANK=str(rank), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+    outs = [p.communicate(timeout=180)[0] for p in procs]
+    for rank, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, out
+        assert f"rank {rank} ok" in out
+
+
 def test_single_process_is_the_identity():
     from paper_2609_39223_b200 import replicas
     assert replicas.world()[0] >= 1
