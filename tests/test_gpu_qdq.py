@@ -362,3 +362,11 @@ def test_tied_tensor_scale_over_fused_projections_and_running_activation_maximum
         assert state.item() == seen and np.float32(s.item()) == np.float32(seen) / np.float32(2688.0)
     zero = api.qf_nvfp4_tensor_scale([torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")], torch.zeros(1, device="cuda"))
     assert zero.item() == 1.0
+    # the steps a row-sharded weight takes: maximum of each shard without a scale, the maxima combined (here by hand, across
+    # ranks by a MAX all-reduce), and the combined state turned into the scale by a call that is given no tensor at all
+    a_state, b_state = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+    assert api.qf_nvfp4_tensor_scale([cat[:40].cuda()], a_state, want_scale=False) is None
+    api.qf_nvfp4_tensor_scale([cat[40:].cuda()], b_state, want_scale=False)
+    combined = torch.maximum(a_state, b_state)
+    shared = api.qf_nvfp4_tensor_scale([], combined, running=True)
+    assert np.float32(shared.item()) == whole["tensor_scale"]
