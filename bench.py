@@ -427,6 +427,7 @@ def run_ours(args):
         e2e_ms = replicas.max_over_ranks(first.elapsed_time(last), dev)
         e2e = {"value": world * FLOP_PER_STEP * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "pcie_gbs_both_directions": (h2d + d2h) * e2e_steps / (e2e_ms * 1e-3) / 1e9,
                "how": "pinned host buffers; upload, kernels and download on three streams, two device buffer sets"}
         del bufs
 
