@@ -31,6 +31,20 @@ def test_no_torch_or_cxx_types_in_the_header():
     assert 'extern "C"' in HEADER
 
 
+def test_header_is_plain_c99(tmp_path):
+    """The boundary is a C ABI: the header must compile as strict C99 with nothing but the standard headers."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler on this machine")
+    src = tmp_path / "use_qf.c"
+    src.write_text('#include "qf.h"\nint main(void) { return qf_status_string(QF_OK) != 0 && sizeof(qf_format_t) > 0 ? 0 : 1; }\n')
+    r = subprocess.run([gcc, "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", str(ROOT / "include"), "-fsyntax-only", str(src)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+
+
 def test_version_and_status_strings():
     assert api.lib().qf_version() >= 100
     seen = {api.status_string(c) for c in range(10)}
