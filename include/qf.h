@@ -174,7 +174,9 @@ qf_status_t qf_fq_linear_bwd(const void* dY, const void* X, const void* W, void*
 /* Per-expert variant for mixture-of-experts layers (every expert's latent weights are trained with
  * the same quantization-aware layer). Rows of X are sorted by expert; group_offsets is a device
  * int32[G+1] of segment starts, each a multiple of 128 (the caller pads segments with zero rows;
- * a zero row quantizes to a zero row in every format); rows_padded = group_offsets[G].
+ * a zero row quantizes to a zero row in every format); rows_padded = group_offsets[G]. The table is device
+ * memory, so the host cannot check it: the kernels force every entry to a multiple of 128 in [0, rows_padded],
+ * and a table that breaks the contract gives meaningless but finite results, never an out-of-range access.
  * W is [G,N,K], Y is [rows_padded,N]:  Y[r,:] = X_hat[r,:] . W_hat[g(r)]^T.
  * NVFP4 weights: every expert is its own tensor with its own tensor scale, so w_tscale is an array of G
  * floats (required; read if QF_W_TSCALE_GIVEN, otherwise written). An NVFP4 activation scale is a

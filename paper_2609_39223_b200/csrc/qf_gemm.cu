@@ -91,6 +91,14 @@ __device__ __forceinline__ uint32_t instr_desc() {
 
 // ---- tile bookkeeping ---------------------------------------------------------------------------
 
+// Segment start i of a grouped call. The table lives in device memory, so the host cannot check it: whatever it holds is
+// forced into the form the interface requires (a multiple of 128 inside [0, rows]), so that a bad table can give
+// wrong numbers but never a negative store coordinate or a contraction loop of unbounded length.
+__device__ __forceinline__ int group_off(const KParams& p, int i) {
+  const int bound = static_cast<int>(p.group_mode == 2 ? p.Kc : p.Mo);
+  return min(max(__ldg(p.offs + i), 0), bound) & ~127;
+}
+
 struct Tile {
   int m0, n0;          // output coordinates (rows of A, rows of B)
   int k_begin, k_end;  // contraction range
@@ -131,8 +139,8 @@ __device__ __forceinline__ Tile decode_tile(const KParams& p, int t, bool need_g
     }
     r.b_row_off = lo * static_cast<int>(p.b_group_rows);
   } else if (p.group_mode == 2) {
-    r.k_begin = __ldg(p.offs + g);
-    r.k_end = __ldg(p.offs + g + 1);
+    r.k_begin = group_off(p, g);
+    r.k_end = group_off(p, g + 1);
     r.c_off = static_cast<int64_t>(g) * p.c_group_stride;
     r.group = g;
   }
@@ -567,12 +575,12 @@ __device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum
       const int mid = (lo + hi) >> 1;
       if (cum[mid] <= mt) lo = mid; else hi = mid;
     }
-    r.m0 = __ldg(p.offs + lo) + (mt - cum[lo]) * (2 * BM);
-    r.rows_limit = __ldg(p.offs + lo + 1);
+    r.m0 = group_off(p, lo) + (mt - cum[lo]) * (2 * BM);
+    r.rows_limit = group_off(p, lo + 1);
     r.b_row_off = lo * static_cast<int>(p.b_group_rows);
   } else if (p.group_mode == 2) {
-    r.k_begin = __ldg(p.offs + g);
-    r.k_end = __ldg(p.offs + g + 1);
+    r.k_begin = group_off(p, g);
+    r.k_end = group_off(p, g + 1);
     r.z = g;
   }
   return r;
@@ -678,7 +686,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int g = lane * 8 + j;
-      cnt[j] = g < p.G ? (__ldg(p.offs + g + 1) - __ldg(p.offs + g) + 2 * BM - 1) / (2 * BM) : 0;
+      cnt[j] = g < p.G ? max(group_off(p, g + 1) - group_off(p, g) + 2 * BM - 1, 0) / (2 * BM) : 0;
       sum += cnt[j];
     }
     int incl = sum;

@@ -247,6 +247,29 @@ def test_grouped_randomly_drawn_segments(seed):
         _close(dw, dw_ref, "grouped dW")
 
 
+@pytest.mark.parametrize("table", [[0, 256, 128, 512, 384, 768, 768], [0, 200, 64, 100000, -5, 700, 768], [768, 0, 0, 0, 0, 0, 0]])
+def test_grouped_calls_force_a_malformed_segment_table_into_range(table):
+    """The segment table is device memory the host cannot validate. The kernels force every entry to a multiple
+    of 128 inside [0, rows], so a table that breaks the contract (not monotone, not aligned, out of range)
+    yields numbers that mean nothing but finite ones, no error status, and a context that still works."""
+    E, rows, F, H = 6, 768, 264, 256
+    Xp = synth.randn_bf16((rows, H), 1.0, 61, device="cuda")
+    W = synth.randn_bf16((E, F, H), 0.02, 62, device="cuda")
+    dYp = synth.randn_bf16((rows, F), 1e-3, 63, device="cuda")
+    offs = torch.tensor(table, dtype=torch.int32, device="cuda")
+    fmt = api.FMT_MXFP4
+    ws = api.workspace(api.OP_GROUPED_BWD, rows, F, H, E)
+    y = api.qf_fq_grouped_linear_fwd(Xp, W, offs, fmt, fmt, y_dtype=torch.float32, ws=ws)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp, Xp, W, offs, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    torch.cuda.synchronize()
+    assert api.qf_read_status(ws) == 0
+    assert bool(torch.isfinite(dw).all())
+    # a well-formed call right afterwards is correct
+    good = torch.tensor([0, 128, 256, 384, 512, 640, 768], dtype=torch.int32)
+    y_ref, _, _ = _grouped_reference(Xp.cpu(), W.cpu(), good, fmt, fmt)
+    _close(api.qf_fq_grouped_linear_fwd(Xp, W, good.cuda(), fmt, fmt, y_dtype=torch.float32), y_ref, "Y after a bad table")
+
+
 def test_grouped_empty_expert_gives_zero_dw():
     E, H, F = 3, 256, 256
     offs = torch.tensor([0, 128, 128, 256], dtype=torch.int32)        # expert 1 has no rows
