@@ -453,7 +453,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // tile with one M=256 MMA stream issued by the leader CTA. Each CTA stages only its own 128 rows of A
 // and its own 128 rows (half) of B, so the shared-memory operand traffic per SM is 64 B/clk instead of
 // the 96 B/clk of the one-CTA tile, and each holds its 128 accumulator rows in its own tensor memory.
-//   * both producers' TMA copies complete on the LEADER's full barrier (no multicast is used);
+//   * both producers' TMA copies complete on the LEADER's full barrier (each CTA fetches its own tiles);
 //   * the leader frees a stage / publishes an accumulator with a tcgen05.commit multicast to the same
 //     barrier offset in both CTAs;
 //   * both CTAs' epilogue warps release the accumulator on the leader's barrier (remote arrive).
@@ -502,7 +502,7 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA copy into this CTA's shared memory whose completion is counted on a barrier that may live in the
-// other CTA of the pair (cluster address). No multicast.
+// other CTA of the pair (cluster address). Each CTA fetches its own tiles; nothing is broadcast.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
