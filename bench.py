@@ -330,6 +330,28 @@ def run_ours(args):
             gbs = Wq.numel() * bytes_per_elem / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
             qdq[name] = {"gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
                          "frac_of_8000_nominal": round(gbs / 8000.0, 4), "bytes_per_elem": bytes_per_elem}
+        # NVFP4 with a speculated tensor scale (QF_TENSOR_SCALE_SPECULATIVE): the scale of the previous call as the guess
+        # (the steady state of a weight in training: a hit), and a zeroed guess before every call (a miss every time)
+        sc = torch.empty(api.scales_shape(api.FMT_NVFP4, *Wq.shape), dtype=torch.uint8, device=dev)
+        carried = torch.zeros(1, dtype=torch.float32, device=dev)
+
+        def spec_hit():
+            api.qf_qdq(api.FMT_NVFP4, Wq, out=out, codes=codes, scales=sc, ws=wsq, tensor_scale=carried, flags=api.TENSOR_SCALE_SPECULATIVE)
+
+        def spec_miss():
+            carried.zero_()
+            spec_hit()
+        for name, fn in (("nvfp4_speculated_scale_hit", spec_hit), ("nvfp4_speculated_scale_miss", spec_miss)):
+            for _ in range(3):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(10):
+                fn()
+            b.record(); torch.cuda.synchronize()
+            gbs = Wq.numel() * 4.5625 / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
+            qdq[name] = {"gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                         "frac_of_8000_nominal": round(gbs / 8000.0, 4), "bytes_per_elem": 4.5625}
         del Wq, out, codes
 
     # ---- headline: K steps, inputs resident in HBM -------------------------------------------------

@@ -81,6 +81,15 @@ typedef enum {
                                       shared-exponent convention of the MX formats. Blocks whose maximum exceeds
                                       3.5 * 2^126 overflow to infinity under this rule. Other formats ignore the flag. */
 
+#define QF_TENSOR_SCALE_SPECULATIVE 0x200u /* qf_qdq, NVFP4, scale not given: *tensor_scale holds a GUESS on entry (for        */
+#define QF_W_TSCALE_SPECULATIVE 0x200u    /* a weight in training: the scale of the previous step). The call quantizes with  */
+                                          /* the guess while it accumulates the true maximum, then derives the scale, stores */
+                                          /* it in *tensor_scale and requantizes unless it equals the guess bit for bit.     */
+                                          /* Results are always those of deriving the scale (Section 3.2.3: the tensor scale */
+                                          /* comes from the current maximum); a right guess saves the separate pass that     */
+                                          /* reads the tensor for its maximum, a wrong one costs a wasted quantize pass.     */
+                                          /* Linear calls: the same for *w_tscale (single weight tensors, not grouped).      */
+
 const char* qf_status_string(qf_status_t s);
 int qf_version(void);
 

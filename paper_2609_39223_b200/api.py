@@ -20,6 +20,7 @@ W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x
 REUSE_W_HAT, REUSE_X_HAT = 0x20, 0x40
 MXFP4_NO_CLIP = 0x80
 SCALES_TILED = 0x100
+TENSOR_SCALE_SPECULATIVE = W_TSCALE_SPECULATIVE = 0x200
 BLOCK = {FMT_NVFP4: 16, FMT_MXFP4: 32, FMT_Q4_K: 256}
 FORMATS = {"none": FMT_NONE, "nvfp4": FMT_NVFP4, "mxfp4": FMT_MXFP4, "q4_k": FMT_Q4_K}
 
@@ -171,12 +172,14 @@ def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_sc
         codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
     if want_scales and scales is None:
         scales = torch.empty(scales_shape(fmt, rows, cols), dtype=torch.uint8, device=dev)
-    flags &= MXFP4_NO_CLIP
+    speculative = bool(flags & TENSOR_SCALE_SPECULATIVE)
+    flags &= MXFP4_NO_CLIP | TENSOR_SCALE_SPECULATIVE
     ts = None
     if fmt == FMT_NVFP4:
         if tensor_scale is not None:
             ts = tensor_scale if isinstance(tensor_scale, torch.Tensor) else torch.tensor([tensor_scale], dtype=torch.float32, device=dev)
-            flags |= TENSOR_SCALE_GIVEN
+            if not speculative:                      # speculative: the tensor holds a guess and receives the derived scale
+                flags |= TENSOR_SCALE_GIVEN
         else:
             ts = ts_out if ts_out is not None else torch.empty(1, dtype=torch.float32, device=dev)
     if ws is None:

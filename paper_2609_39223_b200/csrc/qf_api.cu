@@ -64,7 +64,7 @@ Workspace carve(void* ws, int64_t N, int64_t K, int64_t groups) {
 // array of `groups` floats (required).
 qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t cols, void* dst, float* tscale_user,
                              bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st,
-                             int groups = 1, bool mxfp4_noclip = false) {
+                             int groups = 1, bool mxfp4_noclip = false, bool speculative = false) {
   QdqArgs q{};
   q.mxfp4_noclip = mxfp4_noclip;
   q.fmt = fmt;
@@ -79,6 +79,7 @@ qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t col
       q.tscale_in = tscale_user;
     } else {
       q.tscale_out = tscale_user ? tscale_user : reinterpret_cast<float*>(header + scale_word);
+      if (speculative && tscale_user && groups == 1) return cu(launch_qdq_nvfp4_speculative(q, header, amax_word, kWsGuessW, st));
       return cu(launch_qdq_nvfp4_derive(q, header, amax_word, st));
     }
   }
@@ -139,7 +140,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   if (K > 0) {
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
       if (!(flags & QF_REUSE_W_HAT))
-        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
       Wh = w.w_hat;
     }
     if (a_amax_out) {
@@ -193,7 +194,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     const void* Wh = W;
     if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
       if (!(flags & QF_REUSE_W_HAT))
-        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
+        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
       Wh = w.w_hat;
     }
     g.B = Wh;
@@ -301,6 +302,7 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
       uint32_t* header = static_cast<uint32_t*>(workspace);
       if (cudaError_t e = cudaMemsetAsync(header, 0, kWsHeader, st)) return cu(e);
       q.tscale_out = tensor_scale;
+      if ((flags & QF_TENSOR_SCALE_SPECULATIVE) && tensor_scale) return cu(launch_qdq_nvfp4_speculative(q, header, kWsAmaxW, kWsGuessW, st));
       return cu(launch_qdq_nvfp4_derive(q, header, kWsAmaxW, st));
     } else {
       q.tscale_in = tensor_scale;

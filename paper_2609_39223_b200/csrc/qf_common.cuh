@@ -22,6 +22,7 @@ enum WsWord : int {
   kWsAmaxA = 5,       // max|X|
   kWsScaleW = 8,      // derived NVFP4 tensor scale of W (float)
   kWsScaleA = 9,      // derived NVFP4 tensor scale of X (float)
+  kWsGuessW = 10,     // the caller's guess of W's tensor scale (float bits), kept for the conditional second pass
 };
 
 // ---- device helpers -----------------------------------------------------------------------
@@ -117,6 +118,14 @@ __device__ __forceinline__ uint32_t mxfp4_qdq_pair_bf16(uint32_t w, uint32_t one
 
 // ---- host-side launchers implemented in the .cu files ---------------------------------------
 
+// NVFP4 with a speculated tensor scale: the first pass quantizes with the caller's guess while it accumulates the true
+// maximum; the second pass derives the scale from that maximum and does nothing when it equals the guess.
+struct Nvfp4Speculation {
+  uint32_t* amax_accum;          // first pass: where the maximum of everything read is accumulated (FP32 bits)
+  uint32_t* guess_out;           // first pass: receives the bits of the scale it used
+  const uint32_t* skip_guess;    // second pass: leave at once if the derived scale has these bits
+};
+
 struct QdqArgs {
   int fmt;
   const void* in;
@@ -130,6 +139,7 @@ struct QdqArgs {
   bool reverse;                  // walk the tensor back to front (after an amax pass: L2 holds the tail)
   bool mxfp4_noclip;             // MXFP4: smallest block exponent without saturation (QF_MXFP4_NO_CLIP)
   int groups;                    // NVFP4: > 1 = that many equal tensors back to back, each with its own tensor scale
+  Nvfp4Speculation spec;         // all null unless launch_qdq_nvfp4_speculative() fills it in
   // LoRA merge ahead of the quantizer (lora_rank > 0): the input is W + lora_scale * B A, formed on the fly
   const void* lora_B;            // [rows, rank] BF16
   const void* lora_A;            // [rank, cols] BF16
@@ -138,6 +148,7 @@ struct QdqArgs {
 };
 
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);
+cudaError_t launch_qdq_nvfp4_speculative(const QdqArgs& a, uint32_t* header, int amax_word, int guess_word, cudaStream_t st);
 cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStream_t st);
 cudaError_t launch_amax_to_scale(const uint32_t* amax_bits, float* scale, cudaStream_t st);
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st);

@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
                                                            uint8_t* __restrict__ scales,
                                                            const float* __restrict__ tscale_in,
                                                            const uint32_t* __restrict__ amax_bits,
-                                                           float* __restrict__ tscale_out, int opts) {
+                                                           float* __restrict__ tscale_out, int opts, Nvfp4Speculation spec) {
   const bool reverse = (opts & 1) != 0;       // walk back to front
   const bool noclip = (opts & 2) != 0;        // MXFP4 scale rule without saturation
   // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
@@ -262,9 +262,12 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
     if (amax_bits) {
       const float amax_t = __uint_as_float(amax_bits[blockIdx.y]);
       s_t = amax_t == 0.0f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);            // 2688 = 6 * 448
+      // the first pass already quantized with exactly this scale: nothing to redo (every CTA decides alike)
+      if (spec.skip_guess && __float_as_uint(s_t) == *spec.skip_guess) return;
       if (tscale_out && blockIdx.x == 0 && threadIdx.x == 0) tscale_out[blockIdx.y] = s_t;
     } else {
       s_t = tscale_in[blockIdx.y];
+      if (spec.guess_out && blockIdx.x == 0 && threadIdx.x == 0) *spec.guess_out = __float_as_uint(s_t);
     }
     denom = __fmul_rn(6.0f, s_t);
     denom_safe = div_safe(denom);
@@ -275,6 +278,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
   const int lane = threadIdx.x & 31;
   const int64_t warp_first = first - lane;                    // warp-uniform trip count (shuffles below)
   const int64_t nunits_up = (nunits + 31) & ~static_cast<int64_t>(31);
+  uint32_t seen = 0;                                          // largest block maximum this thread met (speculative first pass)
   for (int64_t base = 0; warp_first + base < nunits_up; base += kUnitsPerThread * stride) {
     uint4 v[kUnitsPerThread][2];
     bool ok[kUnitsPerThread];
@@ -300,6 +304,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
         r = mxfp4_unit(w, m, noclip, scale_code);
       } else {
+        seen = max(seen, m);
         const float amax_b = __uint_as_float(m << 16);
         // quotients near the bottom of the FP32 range take the IEEE divide (warp-uniform choice)
         const bool fast_ok = denom_safe && (amax_b == 0.0f || amax_b >= 0x1p-60f);
@@ -317,6 +322,19 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
           else if ((threadIdx.x & 1) == 0) scales[i >> 1] = static_cast<uint8_t>(scale_code);
         }
       }
+    }
+  }
+  if (FMT == QF_FMT_NVFP4 && spec.amax_accum) {
+    // the true tensor maximum, for the pass that checks the guess (padding lanes contributed zeros)
+    seen = __reduce_max_sync(0xFFFFFFFFu, seen);
+    __shared__ uint32_t warp_seen[kThreads / 32];
+    if (lane == 0) warp_seen[threadIdx.x >> 5] = seen;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t m = 0;
+#pragma unroll
+      for (int k = 0; k < kThreads / 32; ++k) m = max(m, warp_seen[k]);
+      if (m) atomicMax(spec.amax_accum, m << 16);             // BF16 bits -> FP32 bits
     }
   }
 }
@@ -651,12 +669,12 @@ static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStrea
     if (slices > 1 && gx > (kNumSMs * 16 + slices - 1) / slices) gx = (kNumSMs * 16 + slices - 1) / slices;
     qdq_fp4_kernel<QF_FMT_NVFP4, Loader><<<dim3(gx, slices), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), a.tscale_in, a.amax_bits, a.tscale_out,
-        a.reverse ? 1 : 0);
+        a.reverse ? 1 : 0, a.spec);
   } else if (a.fmt == QF_FMT_MXFP4) {
     const int64_t nunits = nelem / 16;
     qdq_fp4_kernel<QF_FMT_MXFP4, Loader><<<capped_grid(nunits, kUnitsPerThread, 0), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr,
-        a.mxfp4_noclip ? 2 : 0);
+        a.mxfp4_noclip ? 2 : 0, Nvfp4Speculation{});
   } else {
     const int64_t nsub = nelem / 32;
     qdq_q4k_kernel<Loader><<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes),
@@ -709,6 +727,28 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
   }
   q.amax_bits = amax_bits;
   return launch_qdq(q, st);
+}
+
+// NVFP4 with a guessed tensor scale in *a.tscale_out (say, the scale of the previous training step). Pass one quantizes
+// with the guess and accumulates the true maximum on the way; pass two derives the scale from that maximum, writes it
+// to *a.tscale_out and requantizes, unless it equals the guess bit for bit, in which case its CTAs return at once.
+// The results are those of deriving the scale first, always; a right guess saves the separate read of the tensor.
+// `header` must have been zeroed on the stream beforehand.
+cudaError_t launch_qdq_nvfp4_speculative(const QdqArgs& a, uint32_t* header, int amax_word, int guess_word, cudaStream_t st) {
+  if (a.groups > 1 || a.lora_rank > 0 || !a.tscale_out) return launch_qdq_nvfp4_derive(a, header, amax_word, st);
+  QdqArgs first = a;
+  first.tscale_in = a.tscale_out;
+  first.tscale_out = nullptr;
+  first.amax_bits = nullptr;
+  first.reverse = false;
+  first.spec = Nvfp4Speculation{header + amax_word, header + guess_word, nullptr};
+  if (cudaError_t e = launch_qdq(first, st)) return e;
+  QdqArgs second = a;
+  second.tscale_in = nullptr;
+  second.amax_bits = header + amax_word;
+  second.reverse = true;
+  second.spec = Nvfp4Speculation{nullptr, nullptr, header + guess_word};
+  return launch_qdq(second, st);
 }
 
 cudaError_t launch_selftest_mxfp4_bf16(unsigned long long* mismatches, cudaStream_t st) {

@@ -472,6 +472,28 @@ def test_independent_calls_on_two_streams():
             assert api.qf_read_status(wss[i]) == 0
 
 
+def test_speculated_weight_scale_through_the_layer():
+    """QF_W_TSCALE_SPECULATIVE in the linear calls: the weight's tensor scale carried from call to call as the next
+    guess. First call (guess 0) misses, later ones hit, a changed weight misses again; outputs always equal the
+    default path's bit for bit and w_tscale always ends up exact."""
+    M, N, K = 384, 520, 1024
+    c = synth.linear_case(M, N, K, seed=77, outlier_channels=2, device="cuda")
+    wq, aq = api.FMT_NVFP4, api.FMT_NONE
+    wts = torch.zeros(1, device="cuda")
+    W = c.W.clone()
+    for step in range(4):
+        if step == 2:
+            W[5, 7] = 3.0                                          # the weight changes: last step's scale is now wrong
+        ref_ts = torch.zeros(1, device="cuda")
+        y0 = api.qf_fq_linear_fwd(c.X, W, wq, aq, y_dtype=torch.float32, w_tscale=ref_ts)
+        dx0, dw0 = api.qf_fq_linear_bwd(c.dY, c.X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, w_tscale=ref_ts)
+        y1 = api.qf_fq_linear_fwd(c.X, W, wq, aq, y_dtype=torch.float32, w_tscale=wts, flags=api.W_TSCALE_SPECULATIVE)
+        dx1, dw1 = api.qf_fq_linear_bwd(c.dY, c.X, W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, w_tscale=wts,
+                                        flags=api.W_TSCALE_SPECULATIVE)
+        assert wts.item() == ref_ts.item()
+        assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     """A device-side wait that can never be satisfied must expire, report QF_ERR_TIMEOUT through the
     status word and leave the context usable (no trap, no hang)."""

@@ -149,6 +149,33 @@ def test_amax_over_odd_lengths_and_negative_maxima():
     assert state.item() == 99.0 and np.float32(scale.item()) == np.float32(99.0) / np.float32(2688.0)
 
 
+@pytest.mark.parametrize("shape", [(64, 512), (129, 2304), (1024, 8192)])
+def test_nvfp4_speculative_tensor_scale_hit_and_miss(shape):
+    """QF_TENSOR_SCALE_SPECULATIVE: whatever the guess, the outputs and the returned scale are those of deriving
+    the scale from the tensor; a wrong guess is corrected by the second pass, a right one leaves the first pass's
+    results in place (the output buffers are poisoned before each call to prove who wrote them)."""
+    xb = torch_to_bits(synth.weight_with_outliers(*shape, seed=shape[0]))
+    x = bits_to_torch(xb, "cuda")
+    o = oracle.qdq(api.FMT_NVFP4, xb)
+    out = torch.empty_like(x); codes = torch.empty((shape[0], shape[1] // 2), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((shape[0], shape[1] // 16), dtype=torch.uint8, device="cuda")
+    exact = float(o["tensor_scale"])
+    for guess in (1.0, 0.0, -3.0, float("nan"), exact * 2, exact, exact):            # misses, then two hits in a row
+        ts = torch.tensor([guess], dtype=torch.float32, device="cuda")
+        out.fill_(-7.0); codes.fill_(0xEE); scales.fill_(0xEE)
+        api.qf_qdq(api.FMT_NVFP4, x, tensor_scale=ts, out=out, codes=codes, scales=scales, flags=api.TENSOR_SCALE_SPECULATIVE)
+        torch.cuda.synchronize()
+        assert np.float32(ts.item()).tobytes() == np.float32(exact).tobytes()
+        np.testing.assert_array_equal(torch_to_bits(out), o["out"])
+        np.testing.assert_array_equal(codes.cpu().numpy(), o["codes"])
+        np.testing.assert_array_equal(scales.cpu().numpy(), o["scales"])
+    # an all-zero tensor derives the scale 1.0
+    z = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    ts = torch.tensor([1.0], dtype=torch.float32, device="cuda")
+    r = api.qf_qdq(api.FMT_NVFP4, z, tensor_scale=ts, flags=api.TENSOR_SCALE_SPECULATIVE)
+    assert ts.item() == 1.0 and not r["out"].any()
+
+
 def test_nvfp4_exact_ties_and_given_scale():
     # with s_t = 2^-10 and a block maximum of 2.625 the block scale is 448 and S = 7/16, so these
     # inputs sit exactly on the rounding midpoints 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5 (times S)
