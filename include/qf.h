@@ -116,7 +116,9 @@ qf_status_t qf_read_status(const void* workspace, void* stream, int* host_status
  *                (scale, offset) pairs}, [rows, cols/256]              (nullable)
  *   tensor_scale NVFP4 only, device float*: read if flags & QF_TENSOR_SCALE_GIVEN, otherwise
  *                written with amax(in)/(6*448) (1.0 for an all-zero tensor). Required for NVFP4.
- * At least one of out_bf16 / codes / scales must be non-NULL. rows*cols == 0 is a no-op. */
+ * At least one of out_bf16 / codes / scales must be non-NULL. rows*cols == 0 is a no-op.
+ * out_bf16 may be the same pointer as in (quantize-dequantize in place); no other overlap between the
+ * buffers is allowed. */
 qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, void* out_bf16,
                    void* codes, void* scales, float* tensor_scale, uint32_t flags, void* workspace,
                    size_t workspace_bytes, void* stream);

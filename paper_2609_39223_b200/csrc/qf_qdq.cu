@@ -735,7 +735,8 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
 // The results are those of deriving the scale first, always; a right guess saves the separate read of the tensor.
 // `header` must have been zeroed on the stream beforehand.
 cudaError_t launch_qdq_nvfp4_speculative(const QdqArgs& a, uint32_t* header, int amax_word, int guess_word, cudaStream_t st) {
-  if (a.groups > 1 || a.lora_rank > 0 || !a.tscale_out) return launch_qdq_nvfp4_derive(a, header, amax_word, st);
+  // (in place, the first pass would destroy the input the second one may need: derive the scale first then)
+  if (a.groups > 1 || a.lora_rank > 0 || !a.tscale_out || a.out == a.in) return launch_qdq_nvfp4_derive(a, header, amax_word, st);
   QdqArgs first = a;
   first.tscale_in = a.tscale_out;
   first.tscale_out = nullptr;

@@ -169,6 +169,12 @@ def test_nvfp4_speculative_tensor_scale_hit_and_miss(shape):
         np.testing.assert_array_equal(torch_to_bits(out), o["out"])
         np.testing.assert_array_equal(codes.cpu().numpy(), o["codes"])
         np.testing.assert_array_equal(scales.cpu().numpy(), o["scales"])
+    # in place (out = in) the guess is not used: the first pass would overwrite what the second needs
+    ts = torch.tensor([exact * 2], dtype=torch.float32, device="cuda")
+    xin = x.clone()
+    api.qf_qdq(api.FMT_NVFP4, xin, tensor_scale=ts, out=xin, want_codes=False, want_scales=False, flags=api.TENSOR_SCALE_SPECULATIVE)
+    np.testing.assert_array_equal(torch_to_bits(xin), o["out"])
+    assert np.float32(ts.item()) == np.float32(exact)
     # an all-zero tensor derives the scale 1.0
     z = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
     ts = torch.tensor([1.0], dtype=torch.float32, device="cuda")
@@ -269,6 +275,19 @@ def test_two_runs_are_bitwise_identical(fmt, name):
     b = api.qf_qdq(fmt, x)
     for k in ("out", "codes", "scales"):
         assert torch.equal(a[k], b[k])
+
+
+@pytest.mark.parametrize("fmt,name", FMTS)
+def test_in_place(fmt, name):
+    """out = in: every thread has read all it needs of its blocks before it writes them."""
+    xb = torch_to_bits(synth.weight_with_outliers(257, 2304 if fmt != api.FMT_Q4_K else 2048, seed=12))
+    o = oracle.qdq(fmt, xb)
+    x = bits_to_torch(xb, "cuda")
+    g = api.qf_qdq(fmt, x, out=x)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(torch_to_bits(x), o["out"])
+    np.testing.assert_array_equal(g["codes"].cpu().numpy(), o["codes"])
+    np.testing.assert_array_equal(g["scales"].cpu().numpy(), o["scales"])
 
 
 def test_optional_outputs_and_empty_tensor():
