@@ -166,7 +166,8 @@ qf_status_t qf_nvfp4_tensor_scale(const void* const* tensors, const int64_t* siz
  *   N a multiple of 8.
  *   w_tscale / a_tscale: NVFP4 tensor scales (device float*), given or derived per flags
  *   (derived values are written back); ignored for other formats and may then be NULL.
- *   a_amax_out (nullable): receives amax(X), for the trainer's running activation maximum. */
+ *   a_amax_out (nullable): receives amax(X), for the trainer's running activation maximum (taken from the
+ *              pass that quantizes X where there is one, so it costs no extra read of X then). */
 qf_status_t qf_fq_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y_dtype, int64_t M, int64_t N,
                              int64_t K, qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale,
                              float* a_tscale, float* a_amax_out, uint32_t flags, void* workspace,

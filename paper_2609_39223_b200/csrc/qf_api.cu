@@ -64,9 +64,10 @@ Workspace carve(void* ws, int64_t N, int64_t K, int64_t groups) {
 // array of `groups` floats (required).
 qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t cols, void* dst, float* tscale_user,
                              bool tscale_given, uint32_t* header, int amax_word, int scale_word, cudaStream_t st,
-                             int groups = 1, bool mxfp4_noclip = false, bool speculative = false) {
+                             int groups = 1, bool mxfp4_noclip = false, bool speculative = false, uint32_t* amax_accum = nullptr) {
   QdqArgs q{};
   q.mxfp4_noclip = mxfp4_noclip;
+  q.spec.amax_accum = amax_accum;       // FP4 formats, single pass: also accumulate max|src| there (zeroed beforehand)
   q.fmt = fmt;
   q.in = src;
   q.rows = rows;
@@ -143,15 +144,22 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
         if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
       Wh = w.w_hat;
     }
-    if (a_amax_out) {
-      if (cudaError_t e = launch_amax(X, M * K, w.header + 6, st)) return cu(e);
-      if (cudaError_t e = launch_amax_to_float(w.header + 6, a_amax_out, st)) return cu(e);
-    }
+    // max|X| for the caller's running maximum: taken from the quantize pass over X where there is one (its own
+    // accumulator for a single-pass FP4 quantizer, the derive path's maximum word for NVFP4 without a supplied
+    // scale), otherwise from a pass of its own
+    const bool x_pass = aq != QF_FMT_NONE && !g.fuse_a_mxfp4 && !(flags & QF_REUSE_X_HAT);
+    const bool x_derives = x_pass && aq == QF_FMT_NVFP4 && !(flags & QF_A_TSCALE_GIVEN);
+    const bool x_accumulates = x_pass && !x_derives && (aq == QF_FMT_NVFP4 || aq == QF_FMT_MXFP4);
+    uint32_t* amax_word = a_amax_out ? (x_derives ? w.header + kWsAmaxA : w.header + 6) : nullptr;
+    if (a_amax_out && !x_derives && !x_accumulates)
+      if (cudaError_t e = launch_amax(X, M * K, amax_word, st)) return cu(e);
     if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
       if (!(flags & QF_REUSE_X_HAT))
-        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
+        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0, false, (a_amax_out && x_accumulates) ? amax_word : nullptr)) return s;
       Xh = w.x_hat;
     }
+    if (a_amax_out)
+      if (cudaError_t e = launch_amax_to_float(amax_word, a_amax_out, st)) return cu(e);
   }
   g.A = Xh; g.B = Wh;
   return cu(launch_gemm(g, st));

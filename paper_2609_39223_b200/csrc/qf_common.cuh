@@ -121,7 +121,8 @@ __device__ __forceinline__ uint32_t mxfp4_qdq_pair_bf16(uint32_t w, uint32_t one
 // NVFP4 with a speculated tensor scale: the first pass quantizes with the caller's guess while it accumulates the true
 // maximum; the second pass derives the scale from that maximum and does nothing when it equals the guess.
 struct Nvfp4Speculation {
-  uint32_t* amax_accum;          // first pass: where the maximum of everything read is accumulated (FP32 bits)
+  uint32_t* amax_accum;          // where the maximum of everything read is accumulated (FP32 bits); also used on its own,
+                                 // by either FP4 format, to report max|x| from the quantize pass
   uint32_t* guess_out;           // first pass: receives the bits of the scale it used
   const uint32_t* skip_guess;    // second pass: leave at once if the derived scale has these bits
 };

@@ -300,11 +300,11 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
       uint32_t m = unit_amax_bits(w);
       uint32_t scale_code;
       UnitOut r;
+      seen = max(seen, m);
       if (FMT == QF_FMT_MXFP4) {
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
         r = mxfp4_unit(w, m, noclip, scale_code);
       } else {
-        seen = max(seen, m);
         const float amax_b = __uint_as_float(m << 16);
         // quotients near the bottom of the FP32 range take the IEEE divide (warp-uniform choice)
         const bool fast_ok = denom_safe && (amax_b == 0.0f || amax_b >= 0x1p-60f);
@@ -324,8 +324,9 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
       }
     }
   }
-  if (FMT == QF_FMT_NVFP4 && spec.amax_accum) {
-    // the true tensor maximum, for the pass that checks the guess (padding lanes contributed zeros)
+  if (spec.amax_accum) {
+    // the maximum of everything this pass read (padding lanes contributed zeros): for the pass that checks a
+    // guessed tensor scale, or for a caller that wants max|x| reported without a separate read
     seen = __reduce_max_sync(0xFFFFFFFFu, seen);
     __shared__ uint32_t warp_seen[kThreads / 32];
     if (lane == 0) warp_seen[threadIdx.x >> 5] = seen;
@@ -674,7 +675,7 @@ static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStrea
     const int64_t nunits = nelem / 16;
     qdq_fp4_kernel<QF_FMT_MXFP4, Loader><<<capped_grid(nunits, kUnitsPerThread, 0), kThreads, 0, st>>>(
         in, nunits, out, static_cast<uint2*>(a.codes), static_cast<uint8_t*>(a.scales), nullptr, nullptr, nullptr,
-        a.mxfp4_noclip ? 2 : 0, Nvfp4Speculation{});
+        a.mxfp4_noclip ? 2 : 0, Nvfp4Speculation{a.spec.amax_accum, nullptr, nullptr});
   } else {
     const int64_t nsub = nelem / 32;
     qdq_q4k_kernel<Loader><<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes),

@@ -121,6 +121,18 @@ def test_nvfp4_scales_written_back_and_amax_reported():
     assert wts.item() == np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.W))["tensor_scale"])
     assert ats.item() == np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.X))["tensor_scale"])
     assert amax.item() == c.X.abs().max().item()
+    # max|X| is reported whichever way the activations are handled (from the quantize pass where there is one)
+    want = c.X.abs().max().item()
+    running = torch.tensor([float(ats.item()) * 1.5], device="cuda")
+    ws = api.workspace(api.OP_LINEAR_BWD, 256, 256, 256)
+    y_ref = api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_MXFP4, y_dtype=torch.float32)
+    for aq, flags, ats_in in ((api.FMT_NVFP4, api.A_TSCALE_GIVEN, running), (api.FMT_MXFP4, 0, None), (api.FMT_NONE, 0, None),
+                              (api.FMT_MXFP4, api.FUSED_QDQ, None), (api.FMT_MXFP4, api.REUSE_X_HAT, None)):
+        amax.fill_(-1.0)
+        y = api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, aq, a_tscale=ats_in, a_amax_out=amax, flags=flags, ws=ws, y_dtype=torch.float32)
+        assert amax.item() == want, (aq, flags)
+        if aq == api.FMT_MXFP4:
+            assert torch.equal(y, y_ref)                  # (the reuse case finds the previous iteration's copy of X_hat)
     # a supplied (tied / running) scale is honoured
     given = torch.tensor([float(wts.item()) * 2], device="cuda")
     y = api.qf_fq_linear_fwd(X, W, api.FMT_NVFP4, api.FMT_NONE, w_tscale=given, flags=api.W_TSCALE_GIVEN, y_dtype=torch.float32)
