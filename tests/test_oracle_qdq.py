@@ -326,6 +326,28 @@ def test_q4k_worked_constant_subblocks():
         assert np.all(out[0, b * 32:(b + 1) * 32] == float(xh[0]))
 
 
+def test_q4k_worked_ramp_superblock():
+    """A whole super-block with eight different sub-block ranges, worked by hand in the golden file."""
+    x = np.zeros((1, 256), np.float32)
+    for b in range(8):
+        x[0, b * 32:(b + 1) * 32] = (b + 1) / 8 * (-1 + 0.125 * (np.arange(32) % 16))
+    xb = f32_to_bits(x)
+    np.testing.assert_array_equal(bits_to_f32(xb), x)                # the inputs are BF16 numbers
+    r = oracle.qdq(FMT_Q4_K, xb)
+    (dh, dminh, s6w, m6w, x0, err), = list(_rows("q4k_worked_ramp.txt"))
+    raw = r["scales"][0, 0]
+    assert int(raw[0]) | int(raw[1]) << 8 == int(dh[0], 16)
+    assert int(raw[2]) | int(raw[3]) << 8 == int(dminh[0], 16)
+    d, dmin, s6, m6 = _q4k_meta(r["scales"])
+    assert list(s6[0, 0]) == [int(v) for v in s6w] and list(m6[0, 0]) == [int(v) for v in m6w]
+    codes = _q4k_codes(r["codes"], 1, 256)[0]
+    np.testing.assert_array_equal(codes[224:], np.tile(np.arange(16), 2))
+    out = bits_to_f32(r["out"])[0]
+    np.testing.assert_array_equal(out[224:], x[0, 224:])
+    assert codes[0] == 0 and out[0] == float(x0[0])
+    assert np.abs(out - x[0]).max() == float(err[0])
+
+
 def test_q4k_record_reads_back_through_gguf():
     from gguf import GGMLQuantizationType as T, quants
     rows, cols = 8, 1024

@@ -1,5 +1,7 @@
 """Engine-native packing (the export / weight-synchronisation step): oracle pins on CPU, and the CUDA
 re-layout kernels against the oracle, byte for byte."""
+from pathlib import Path
+
 import numpy as np
 import pytest
 import torch
@@ -8,6 +10,8 @@ import oracle
 from oracle import FMT_MXFP4, FMT_NVFP4, FMT_Q4_K
 from paper_2609_39223_b200 import api, synth
 from util import f32_to_bits, torch_to_bits
+
+GOLDEN = Path(__file__).parent / "golden"
 
 
 def _w(rows, cols, seed):
@@ -43,6 +47,50 @@ def test_oracle_scale_swizzle_is_a_padded_bijection_with_the_documented_tile_lay
             assert z[o] == s[r, c] and not seen[o]
             seen[o] = True
     assert not z[~seen].any()
+
+
+def _tiled_scales_by_reshape(s: np.ndarray) -> np.ndarray:
+    """The tiled scale-factor layout written a second way, from its description as nested blocks rather than as
+    a byte-offset formula (NVIDIA's documentation of 1-D block-scaling factor layouts for block-scaled matmuls:
+    128 x 4 scale tiles, each stored as 32 rows of 16 bytes in which row i holds the four scales of rows
+    i, i + 32, i + 64, i + 96 one after another; tiles follow each other along the scale columns first)."""
+    rows, nblk = s.shape
+    rt, ct = -(-rows // 128), -(-nblk // 4)
+    p = np.zeros((rt * 128, ct * 4), np.uint8)
+    p[:rows, :nblk] = s
+    # [row tile, quarter of the tile (rows 32q..32q+31), row in quarter, column tile, column in tile]
+    return p.reshape(rt, 4, 32, ct, 4).transpose(0, 3, 2, 1, 4).reshape(-1)
+
+
+@pytest.mark.parametrize("rows,nblk", [(1, 1), (128, 4), (130, 6), (200, 10), (257, 33), (384, 128)])
+def test_oracle_scale_swizzle_equals_the_nested_block_description(rows, nblk):
+    rng = np.random.default_rng(rows * 1000 + nblk)
+    s = rng.integers(1, 256, (rows, nblk), dtype=np.uint8)
+    np.testing.assert_array_equal(oracle.swizzle_block_scales(s), _tiled_scales_by_reshape(s))
+
+
+def test_oracle_scale_swizzle_stored_offsets():
+    """Byte offsets of every entry of a 130 x 6 scale matrix, stored by golden/make_fp4_scale_tiles.py; the
+    first tile's first rows are also spelled out here by hand from the layout's description."""
+    table = {}
+    for line in (GOLDEN / "fp4_scale_tiles.txt").read_text().splitlines():
+        if line.strip() and not line.startswith("#"):
+            r, offs = line.split("|")
+            table[int(r)] = [int(v) for v in offs.split()]
+    assert len(table) == 130
+    # by hand: row 0 opens the tile; row 1 is the next 16-byte line; rows 32 / 64 / 96 share line 0 with row 0;
+    # scale columns 4, 5 open the next tile (512 bytes on); row 128 opens the second row of tiles (2 tiles on)
+    assert table[0] == [0, 1, 2, 3, 512, 513] and table[1][:4] == [16, 17, 18, 19]
+    assert table[32][:4] == [4, 5, 6, 7] and table[64][:4] == [8, 9, 10, 11] and table[96][:4] == [12, 13, 14, 15]
+    assert table[127][:4] == [508, 509, 510, 511] and table[128] == [1024, 1025, 1026, 1027, 1536, 1537]
+    s = np.random.default_rng(5).integers(1, 256, (130, 6), dtype=np.uint8)
+    z = oracle.swizzle_block_scales(s)
+    used = np.zeros(z.size, bool)
+    for r, offs in table.items():
+        for c, o in enumerate(offs):
+            assert z[o] == s[r, c]
+            used[o] = True
+    assert used.sum() == 130 * 6 and not z[~used].any()
 
 
 @pytest.mark.gpu
