@@ -2,7 +2,8 @@
  *
  * C ABI of libqf.so. Plain C types only. Unless a parameter says otherwise, EVERY data pointer
  * is a DEVICE pointer owned by the caller; the library never allocates or frees device memory,
- * keeps no state between calls, and enqueues all of its work on the CUDA stream passed as
+ * keeps no state between calls beyond per-device caches of constants (device capability, kernel
+ * attributes, the address of one built-in buffer), and enqueues all of its work on the CUDA stream passed as
  * `stream` (a cudaStream_t cast to void*, NULL = the legacy default stream). Calls return as soon
  * as the work is enqueued. Scratch memory comes from the caller through `workspace` /
  * `workspace_bytes`; qf_workspace_bytes() says how much a call needs.
@@ -177,7 +178,7 @@ qf_status_t qf_fq_linear_fwd(const void* X, const void* W, void* Y, qf_dtype_t y
  *     dX[M,K] = dY[M,N] . W_hat[N,K]            (nullable: skip)
  *     dW[N,K] = dY[M,N]^T . X_hat[M,K]          (nullable: skip)
  * W_hat and X_hat are recomputed from W and X exactly as in the forward. dY is never quantized.
- * M must be a multiple of 8 when dW is requested. */
+ * M may be any size (the contraction of dW needs no padding). */
 qf_status_t qf_fq_linear_bwd(const void* dY, const void* X, const void* W, void* dX, qf_dtype_t dx_dtype,
                              void* dW, qf_dtype_t dw_dtype, int64_t M, int64_t N, int64_t K,
                              qf_format_t wq_fmt, qf_format_t aq_fmt, float* w_tscale, float* a_tscale,
@@ -260,12 +261,19 @@ qf_status_t qf_fp4_matmul_native(qf_format_t fmt, const void* a_codes, const voi
  * library: QF_NOALLOC_SCRATCH_BYTES (32 MiB) of device memory per GPU, held by every GPU that loads
  * libqf.so until the process exits.
  *
- * Same arithmetic, arguments and results as qf_fq_linear_fwd (no a_amax_out, no workspace). The call
- * allocates nothing: no cudaMalloc / cudaFree / allocating library routine on any path.
+ * Same arithmetic, arguments and results as qf_fq_linear_fwd (no a_amax_out, no workspace;
+ * QF_REUSE_W_HAT / QF_REUSE_X_HAT are ignored, since the buffer is shared by every caller). The call
+ * itself allocates nothing: no cudaMalloc / cudaFree / allocating library routine on any path. The
+ * buffer is part of the library's device image; with CUDA's default lazy module loading the driver
+ * places that image on a device the first time something from the library runs there, so the
+ * 32 MiB are taken at that moment (for this entry point: at its first call on the device), not at
+ * dlopen. A host that is about to reserve all remaining device memory should make one call first
+ * (M = 0 is enough), or it will get QF_ERR_CUDA from the first real call.
  *   Limit: 256 + round256(2*N*K) + round256(2*M*K) bytes must fit in QF_NOALLOC_SCRATCH_BYTES; larger
  *          problems are rejected with QF_ERR_TOO_LARGE before anything is enqueued.
  *   First call on each device: looks up the device address of the built-in buffer (once per device,
- *          with that device current). Make that first call outside any stream capture.
+ *          with that device current; this is also what makes the driver load the image, see above).
+ *          Make that first call outside any stream capture.
  *   Sharing: every call on a device uses the same buffer, which keeps the previous call's contents;
  *          the call clears the words that must start at zero itself. Two calls whose GPU work can
  *          overlap (different streams, no dependency between them) race on the buffer — serialise

@@ -1,6 +1,8 @@
 // C ABI of libqf.so: argument validation, workspace carving, and the launch sequences of the
 // quantizer and of the quantization-aware linear layer (forward and straight-through backward).
 // Nothing here computes; every step of the path runs in the kernels of qf_qdq.cu / qf_gemm.cu.
+// The only state kept between calls is per-device caches of facts that never change (compute capability,
+// kernel attributes already set, the device address of the allocation-free entry point's built-in buffer).
 #include <stdio.h>
 
 #include "qf_common.cuh"
@@ -74,7 +76,6 @@ qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t col
   q.cols = cols;
   q.out = dst;
   q.groups = fmt == QF_FMT_NVFP4 ? groups : 1;
-  if (fmt == QF_FMT_NVFP4 && groups > 1 && !tscale_user) return QF_ERR_NULL;
   if (fmt == QF_FMT_NVFP4) {
     if (tscale_given) {
       q.tscale_in = tscale_user;
@@ -100,6 +101,7 @@ qf_status_t check_linear_common(const void* W, bool need_w, int64_t M, int64_t N
   if (wq != QF_FMT_NONE && K % block_of(wq)) return QF_ERR_SHAPE;
   if (aq != QF_FMT_NONE && K % block_of(aq)) return QF_ERR_SHAPE;
   if (wq == QF_FMT_NVFP4 && (flags & QF_W_TSCALE_GIVEN) && !w_ts) return QF_ERR_NULL;
+  if (wq == QF_FMT_NVFP4 && groups > 1 && !w_ts) return QF_ERR_NULL;       // one tensor scale per expert: the array is required
   if (aq == QF_FMT_NVFP4 && (flags & QF_A_TSCALE_GIVEN) && !a_ts) return QF_ERR_NULL;
   if ((W && !aligned16(W)) || !aligned16(ws)) return QF_ERR_ALIGN;
   if (ws_bytes < linear_ws_bytes(M, N, K, groups)) return QF_ERR_WORKSPACE;
@@ -114,12 +116,15 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
                             uint32_t flags, void* ws, size_t ws_bytes, cudaStream_t st) {
   const bool grouped = offs != nullptr;
   const int64_t groups = grouped ? G : 1;
-  if (!X || !Y) return QF_ERR_NULL;
+  const bool has_operands = M != 0 && N != 0 && K != 0;      // empty operands have no storage to point at
+  if ((has_operands && !X) || (M != 0 && N != 0 && !Y)) return QF_ERR_NULL;
   if (!valid_dtype(y_dtype)) return QF_ERR_DTYPE;
-  if (qf_status_t s = check_linear_common(W, true, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
+  if (qf_status_t s = check_linear_common(W, has_operands, M, N, K, wq, aq, w_ts, a_ts, flags, ws, ws_bytes, groups)) return s;
   if (!aligned16(X) || !aligned16(Y)) return QF_ERR_ALIGN;
   if (qf_status_t s = check_arch()) return s;
   if (M == 0 || N == 0) return QF_OK;
+  if (K == 0)        // an empty contraction still defines the output: zeros
+    return cu(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * (y_dtype == QF_DT_F32 ? 4 : 2), st));
   Workspace w = carve(ws, N, K, groups);
   if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
   GemmArgs g{};
@@ -150,7 +155,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
     const bool x_pass = aq != QF_FMT_NONE && !g.fuse_a_mxfp4 && !(flags & QF_REUSE_X_HAT);
     const bool x_derives = x_pass && aq == QF_FMT_NVFP4 && !(flags & QF_A_TSCALE_GIVEN);
     const bool x_accumulates = x_pass && !x_derives && (aq == QF_FMT_NVFP4 || aq == QF_FMT_MXFP4);
-    uint32_t* amax_word = a_amax_out ? (x_derives ? w.header + kWsAmaxA : w.header + 6) : nullptr;
+    uint32_t* amax_word = a_amax_out ? (x_derives ? w.header + kWsAmaxA : w.header + kWsAmaxReport) : nullptr;
     if (a_amax_out && !x_derives && !x_accumulates)
       if (cudaError_t e = launch_amax(X, M * K, amax_word, st)) return cu(e);
     if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
@@ -487,6 +492,8 @@ qf_status_t qf_fq_linear_fwd_noalloc(const void* X, const void* W, void* Y, qf_d
   if (qf_status_t s = check_arch()) return s;
   void* scratch = nullptr;
   if (qf_status_t s = noalloc_scratch_ptr(&scratch)) return s;
+  // the buffer is shared by every caller: copies left there by an earlier call are never trusted
+  flags &= ~static_cast<uint32_t>(QF_REUSE_W_HAT | QF_REUSE_X_HAT);
   return linear_fwd_impl(X, W, Y, y_dtype, nullptr, 1, M, N, K, wq_fmt, aq_fmt, w_tscale, a_tscale, nullptr, flags, scratch,
                          QF_NOALLOC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
 }

@@ -20,6 +20,7 @@ enum WsWord : int {
   kWsStatus = 0,      // qf_status_t written by a device-side wait that gave up
   kWsAmaxW = 4,       // max|W| as FP32 bits (unsigned-integer max is order preserving for x >= 0)
   kWsAmaxA = 5,       // max|X|
+  kWsAmaxReport = 6,  // max|X| gathered for the caller's a_amax_out when the quantize pass over X does not derive a scale
   kWsScaleW = 8,      // derived NVFP4 tensor scale of W (float)
   kWsScaleA = 9,      // derived NVFP4 tensor scale of X (float)
   kWsGuessW = 10,     // the caller's guess of W's tensor scale (float bits), kept for the conditional second pass

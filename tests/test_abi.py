@@ -105,6 +105,8 @@ def test_linear_argument_errors_need_no_gpu():
     assert g(P, P, P, 0, None, 4, 512, N, K, 2, 2, None, None, 0, P, 1 << 30, None) == 1
     assert g(P, P, P, 0, P, 4, 500, N, K, 2, 2, None, None, 0, P, 1 << 30, None) == 2          # rows not padded to 128
     assert g(P, P, P, 0, P, 0, 512, N, K, 2, 2, None, None, 0, P, 1 << 30, None) == 2
+    # grouped NVFP4 weights need the per-expert scale array: refused with the other checks, before anything is enqueued
+    assert g(P, P, P, 0, P, 4, 512, N, K, api.FMT_NVFP4, 0, None, None, 0, P, 1 << 30, None) == 1
 
 
 def test_calls_fail_loudly_without_a_device():

@@ -1,0 +1,179 @@
+"""More GPU parity cases of the quantization-aware layer through the C ABI: the in-kernel quantizer over many
+tiles per CTA pair, NVFP4 on both operands with supplied tensor scales, grouped layers with NVFP4 activations and
+with Q4_K weights, and the down projection of the 32K-token workload at full size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39223_b200 import api, synth
+from util import torch_to_bits
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2          # max|diff| <= 1e-2 * rms(reference), on FP32 outputs
+
+
+def _rms(a):
+    return float(np.sqrt(np.mean(np.square(a.astype(np.float64)))))
+
+
+def _close(got, ref, what):
+    got = got.detach().float().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    err = float(np.abs(got.astype(np.float64) - ref.astype(np.float64)).max())
+    bound = TOL * _rms(ref)
+    assert err <= bound, f"{what}: max|diff| {err:.3e} > {bound:.3e}"
+
+
+# (M, N, K): forward / dX / dW pair tiles and k-blocks per tile
+#   2560 x 2304 x  832: 90 / 40 / 36 tiles, 13 / 36 / 40 k-blocks (13 is not a multiple of the 6-stage ring)
+#   4096 x 8192 x  512: 512 / 32 / 64 tiles (seven per CTA pair in the forward), 8 / 128 / 64 k-blocks
+#   1152 x 4608 x 1280: 90 / 25 / 90 tiles with a half-empty last row tile, 20 / 72 / 18 k-blocks
+MULTI_TILE = [(2560, 2304, 832), (4096, 8192, 512), (1152, 4608, 1280)]
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_MXFP4, api.FMT_NONE), (api.FMT_NONE, api.FMT_MXFP4)])
+@pytest.mark.parametrize("M,N,K", MULTI_TILE)
+def test_in_kernel_quantization_over_many_tiles_per_cta_pair(wq, aq, M, N, K):
+    """With more pair tiles than the 74 CTA pairs of the persistent grid, the in-kernel quantizer's running k-block
+    counter, its stage and phase wrap across tiles, the transform groups running ahead of each other and the
+    double-buffered accumulators are all exercised. Outputs must be the default path's bits, the status word clean,
+    and sampled rows within tolerance of the oracle."""
+    c = synth.linear_case(M, N, K, seed=M + N + K, outlier_channels=4, device="cuda")
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    y0 = api.qf_fq_linear_fwd(c.X, c.W, wq, aq, y_dtype=torch.float32, ws=ws)
+    dx0, dw0 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    y1 = api.qf_fq_linear_fwd(c.X, c.W, wq, aq, y_dtype=torch.float32, flags=api.FUSED_QDQ, ws=ws)
+    dx1, dw1 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32,
+                                    flags=api.FUSED_QDQ, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(y0, y1), "Y"
+    assert torch.equal(dx0, dx1), "dX"
+    assert torch.equal(dw0, dw1), "dW"
+    rng = np.random.default_rng(K)
+    rows = np.sort(rng.choice(M, 12, replace=False)); rows[0] = 0; rows[-1] = M - 1
+    n_idx = np.sort(rng.choice(N, 8, replace=False)); n_idx[0] = 0; n_idx[-1] = N - 1
+    xb, wb, dyb = torch_to_bits(c.X), torch_to_bits(c.W), torch_to_bits(c.dY)
+    w_hat, x_hat = oracle.qdq_out(wq, wb), oracle.qdq_out(aq, xb)
+    _close(y1[rows], oracle.matmul_fwd(x_hat[rows], w_hat), "Y rows")
+    _close(dx1[rows], oracle.matmul_dgrad(dyb[rows], w_hat), "dX rows")
+    _close(dw1[n_idx], oracle.matmul_wgrad(dyb, x_hat, n_idx), "dW rows")
+
+
+@pytest.mark.parametrize("M,N,K", [(200, 264, 768), (520, 776, 1024)])
+def test_nvfp4_on_both_operands_with_supplied_tensor_scales(M, N, K):
+    """NVFP4 weights and activations with both tensor scales handed in (a tied weight scale, a running activation
+    scale): forward and backward against the oracle run with the same two scales, and the scale words left alone."""
+    c = synth.linear_case(M, N, K, seed=N, outlier_channels=2)
+    xb, wb, dyb = (torch_to_bits(t) for t in (c.X, c.W, c.dY))
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    # scales a trainer could hold: 1.5x and 0.75x the ones the current tensors would derive (the second saturates blocks)
+    for fw, fa in ((1.5, 1.5), (0.75, 2.0)):
+        w_ts = np.float32(oracle.qdq(api.FMT_NVFP4, wb)["tensor_scale"]) * np.float32(fw)
+        a_ts = np.float32(oracle.qdq(api.FMT_NVFP4, xb)["tensor_scale"]) * np.float32(fa)
+        wts = torch.tensor([w_ts], dtype=torch.float32, device="cuda")
+        ats = torch.tensor([a_ts], dtype=torch.float32, device="cuda")
+        flags = api.W_TSCALE_GIVEN | api.A_TSCALE_GIVEN
+        y = api.qf_fq_linear_fwd(X, W, api.FMT_NVFP4, api.FMT_NVFP4, y_dtype=torch.float32, w_tscale=wts, a_tscale=ats, flags=flags)
+        dx, dw = api.qf_fq_linear_bwd(dY, X, W, api.FMT_NVFP4, api.FMT_NVFP4, dx_dtype=torch.float32, dw_dtype=torch.float32,
+                                      w_tscale=wts, a_tscale=ats, flags=flags)
+        assert wts.item() == w_ts and ats.item() == a_ts
+        _close(y, oracle.fq_linear_fwd(xb, wb, api.FMT_NVFP4, api.FMT_NVFP4, w_tscale=float(w_ts), a_tscale=float(a_ts)), "Y")
+        dx_ref, dw_ref = oracle.fq_linear_bwd(dyb, xb, wb, api.FMT_NVFP4, api.FMT_NVFP4, w_tscale=float(w_ts), a_tscale=float(a_ts))
+        _close(dx, dx_ref, "dX")
+        _close(dw, dw_ref, "dW")
+        # the supplied scales matter: deriving them gives another result
+        assert not torch.equal(y, api.qf_fq_linear_fwd(X, W, api.FMT_NVFP4, api.FMT_NVFP4, y_dtype=torch.float32))
+
+
+def _segments(counts):
+    offs = torch.zeros(len(counts) + 1, dtype=torch.int32)
+    offs[1:] = torch.cumsum(torch.tensor(counts) * 128, 0)
+    return offs
+
+
+def _grouped_oracle(Xp, W, dYp, offs, wq, aq, w_ts=None, a_ts=None):
+    ys, dxs, dws = [], [], []
+    for g in range(W.shape[0]):
+        a, b = int(offs[g]), int(offs[g + 1])
+        wt = None if w_ts is None else float(w_ts[g])
+        if b > a:
+            xb, wb, dyb = torch_to_bits(Xp[a:b]), torch_to_bits(W[g]), torch_to_bits(dYp[a:b])
+            ys.append(oracle.fq_linear_fwd(xb, wb, wq, aq, w_tscale=wt, a_tscale=a_ts))
+            dx, dw = oracle.fq_linear_bwd(dyb, xb, wb, wq, aq, w_tscale=wt, a_tscale=a_ts)
+        else:
+            dx, dw = np.zeros((0, W.shape[2]), np.float32), np.zeros(tuple(W.shape[1:]), np.float32)
+        dxs.append(dx); dws.append(dw)
+    return np.concatenate(ys), np.concatenate(dxs), np.stack(dws)
+
+
+def test_grouped_layer_with_nvfp4_activations_and_weights():
+    """Grouped call, NVFP4 on both operands: one tensor scale per expert for the weights, a single activation scale
+    for the whole routed input (derived here from all routed rows, then supplied in the backward)."""
+    E, H, F = 5, 512, 264
+    offs = _segments([2, 1, 0, 3, 2])
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 41)
+    W = synth.randn_bf16((E, F, H), 0.02, 42)
+    W = (W.float() * torch.tensor([1.0, 4.0, 0.25, 8.0, 0.5]).view(E, 1, 1)).to(torch.bfloat16)
+    dYp = synth.randn_bf16((rows, F), 1e-3, 43)
+    a_ts = float(oracle.qdq(api.FMT_NVFP4, torch_to_bits(Xp))["tensor_scale"])          # over all routed rows
+    w_ts = [np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(W[g]))["tensor_scale"]) for g in range(E)]
+    y_ref, dx_ref, dw_ref = _grouped_oracle(Xp, W, dYp, offs, api.FMT_NVFP4, api.FMT_NVFP4, w_ts, a_ts)
+    wts, ats = torch.zeros(E, device="cuda"), torch.zeros(1, device="cuda")
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NVFP4, y_dtype=torch.float32,
+                                     w_tscale=wts, a_tscale=ats)
+    assert ats.item() == np.float32(a_ts) and [np.float32(v) for v in wts.cpu().tolist()] == w_ts
+    _close(y, y_ref, "Y")
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_NVFP4, api.FMT_NVFP4,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32, w_tscale=wts, a_tscale=ats,
+                                          flags=api.W_TSCALE_GIVEN | api.A_TSCALE_GIVEN)
+    _close(dx, dx_ref, "dX")
+    _close(dw, dw_ref, "dW")
+
+
+def test_grouped_layer_with_q4k_weights():
+    E, H, F = 4, 512, 264                 # K = 512: two super-blocks per weight row
+    offs = _segments([1, 3, 0, 2])
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 51)
+    W = synth.randn_bf16((E, F, H), 0.02, 52)
+    dYp = synth.randn_bf16((rows, F), 1e-3, 53)
+    y_ref, dx_ref, dw_ref = _grouped_oracle(Xp, W, dYp, offs, api.FMT_Q4_K, api.FMT_NONE)
+    y = api.qf_fq_grouped_linear_fwd(Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_Q4_K, api.FMT_NONE, y_dtype=torch.float32)
+    dx, dw = api.qf_fq_grouped_linear_bwd(dYp.cuda(), Xp.cuda(), W.cuda(), offs.cuda(), api.FMT_Q4_K, api.FMT_NONE,
+                                          dx_dtype=torch.float32, dw_dtype=torch.float32)
+    _close(y, y_ref, "Y"); _close(dx, dx_ref, "dX"); _close(dw, dw_ref, "dW")
+    assert torch.count_nonzero(dw[2]) == 0
+
+
+def test_full_size_nvfp4_weight_only_down_projection_sampled_rows():
+    """The down projection of the 32K-token workload at full size: H 32768 x 14336, W_down 4096 x 14336, NVFP4
+    weights, unquantized activations, forward and both backward products on sampled rows."""
+    M, N, K = 32768, 4096, 14336
+    c = synth.linear_case(M, N, K, seed=5, device="cuda", outlier_channels=0)
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    wts = torch.zeros(1, device="cuda")
+    y = api.qf_fq_linear_fwd(c.X, c.W, api.FMT_NVFP4, api.FMT_NONE, y_dtype=torch.float32, ws=ws, w_tscale=wts)
+    dx, dw = api.qf_fq_linear_bwd(c.dY, c.X, c.W, api.FMT_NVFP4, api.FMT_NONE, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    rng = np.random.default_rng(5)
+    rows = np.sort(rng.choice(M, 12, replace=False)); rows[0] = 0; rows[-1] = M - 1
+    sel = torch.from_numpy(rows).cuda()
+    qw = oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.W))
+    assert wts.item() == np.float32(qw["tensor_scale"])
+    _close(y[sel], oracle.matmul_fwd(torch_to_bits(c.X[sel]), qw["out"]), "Y rows")
+    _close(dx[sel], oracle.matmul_dgrad(torch_to_bits(c.dY[sel]), qw["out"]), "dX rows")
+    n_idx = np.sort(rng.choice(N, 4, replace=False)); n_idx[0] = 0; n_idx[-1] = N - 1
+    dy_cols = torch_to_bits(c.dY[:, torch.from_numpy(n_idx).cuda()].contiguous())        # the 4 columns of dY those rows of dW need
+    dw_ref = oracle.matmul_wgrad(dy_cols, torch_to_bits(c.X))
+    _close(dw[torch.from_numpy(n_idx).cuda()], dw_ref, "dW rows")
+
+
+def test_forward_with_an_empty_contraction_gives_zeros():
+    X = torch.empty((300, 0), dtype=torch.bfloat16, device="cuda")
+    W = torch.empty((264, 0), dtype=torch.bfloat16, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        Y = torch.full((300, 264), float("nan"), dtype=dt, device="cuda")
+        api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_MXFP4, Y=Y)
+        assert torch.count_nonzero(Y) == 0

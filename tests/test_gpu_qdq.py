@@ -314,6 +314,24 @@ def test_full_size_q4k_decoder_matrices(name):
     _compare(api.FMT_Q4_K, torch_to_bits(w))
 
 
+@pytest.mark.parametrize("name", ["q_proj", "v_proj", "o_proj", "gate_proj", "up_proj"])
+def test_full_size_q4k_decoder_matrices_row_slices(name):
+    """The other five linear weights of a decoder layer at full size (per-layer seed): the GPU quantizes the whole
+    matrix, the oracle the first, a middle and the last 48 rows (rows are independent in Q4_K)."""
+    w = synth.dense_decoder_weight(17, name, device="cuda")
+    g = api.qf_qdq(api.FMT_Q4_K, w)
+    rows = w.shape[0]
+    pick = np.concatenate([np.arange(48), rows // 2 + np.arange(48), rows - 48 + np.arange(48)])
+    sel = torch.from_numpy(pick).cuda()
+    o = oracle.qdq(api.FMT_Q4_K, torch_to_bits(w[sel]))
+    np.testing.assert_array_equal(torch_to_bits(g["out"][sel]), o["out"])
+    np.testing.assert_array_equal(g["codes"][sel].cpu().numpy(), o["codes"])
+    np.testing.assert_array_equal(g["scales"][sel].cpu().numpy(), o["scales"])
+    # nothing left unwritten: every row of the dequantized matrix is within one quantization step of its input
+    err = (g["out"].float() - w.float()).abs_().amax(dim=1)
+    assert float(err.max()) <= 0.02 * 6 / 15 and float(err.min()) > 0
+
+
 def test_full_size_mxfp4_activation():
     x = synth.activations_with_outlier_channels(8192, 4096, seed=0)
     _compare(api.FMT_MXFP4, torch_to_bits(x))

@@ -1,18 +1,18 @@
-"""The allocation-free forward entry point (for hosts that may not allocate device memory when they
-call us: the scratch it needs is a fixed buffer inside the library) must give what the ordinary
-entry point gives. Collected last on purpose; passes on its own and after the rest of the suite."""
+"""The allocation-free forward entry point. Some hosts cannot give the library scratch memory when they
+call it: an extension running inside a process whose memory planner took the whole device up front and
+forbids further device allocations, or a loop that must never enter an allocator. For them the two
+transient fake-quantized copies live in a fixed buffer inside the library. The entry point must give
+exactly what the ordinary one gives, call after call, and must leave the amount of free device memory
+untouched. Collected last on purpose; passes on its own and after the rest of the suite."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_39223_b200 import api, synth
+from util import torch_to_bits
 
-TOL = 1e-2          # same bound as the other linear-layer tests: max|diff| <= 1e-2 * rms(reference)
-
-
-def _check_same(got, ref):
-    ref32, got32 = ref.float(), got.float()
-    rms = ref32.pow(2).mean().sqrt().item()
-    assert (got32 - ref32).abs().max().item() <= TOL * rms
+TOL = 1e-2          # the linear-layer bound used everywhere: max|diff| <= 1e-2 * rms(reference)
 
 
 @pytest.mark.gpu
@@ -29,13 +29,43 @@ def test_noalloc_forward_matches_workspace_forward_twice_in_a_row():
             ats = torch.zeros(1, device="cuda") if aq == api.FMT_NVFP4 else None
             api.qf_fq_linear_fwd_noalloc(X, W, Y, wq, aq, w_tscale=wts, a_tscale=ats)
             torch.cuda.synchronize()
-            _check_same(Y, ref)
+            # same kernels, same operands, same summation order: within the tolerance trivially, and in fact identical
+            rms = ref.pow(2).mean().sqrt().item()
+            assert (Y - ref).abs().max().item() <= TOL * rms
+            assert torch.equal(Y, ref)
+            # and against the oracle, like every other path
+            y_ref = oracle.fq_linear_fwd(torch_to_bits(c.X), torch_to_bits(c.W), wq, aq)
+            err = np.abs(Y.cpu().numpy().astype(np.float64) - y_ref).max()
+            assert err <= TOL * np.sqrt(np.mean(np.square(y_ref.astype(np.float64))))
     # BF16 output through the same path
     X, W = c1.X.cuda(), c1.W.cuda()
     ref = api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_NONE)
     Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     api.qf_fq_linear_fwd_noalloc(X, W, Y, api.FMT_MXFP4, api.FMT_NONE)
-    _check_same(Y, ref)
+    assert torch.equal(Y, ref)
+
+
+@pytest.mark.gpu
+def test_noalloc_call_leaves_free_device_memory_unchanged():
+    M, N, K = 512, 768, 1024
+    c = synth.linear_case(M, N, K, seed=23, outlier_channels=1, device="cuda")
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    fmt = api.FMT_MXFP4
+    api.qf_fq_linear_fwd_noalloc(c.X, c.W, Y, fmt, fmt)             # first call on this device: set-up happens here
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    reserved_before = torch.cuda.memory_reserved()
+    for _ in range(3):
+        api.qf_fq_linear_fwd_noalloc(c.X, c.W, Y, fmt, fmt)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before                                 # nothing was taken from (or returned to) the driver
+    assert torch.cuda.memory_reserved() == reserved_before           # nor from torch's caching allocator
+    # copies a previous caller left in the shared buffer are never trusted: the reuse flags are ignored
+    c2 = synth.linear_case(M, N, K, seed=24, outlier_channels=1, device="cuda")
+    Y2 = torch.empty_like(Y)
+    api.qf_fq_linear_fwd_noalloc(c2.X, c2.W, Y2, fmt, fmt, flags=api.REUSE_W_HAT | api.REUSE_X_HAT)
+    assert torch.equal(Y2, api.qf_fq_linear_fwd(c2.X, c2.W, fmt, fmt))
 
 
 @pytest.mark.gpu
