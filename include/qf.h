@@ -57,7 +57,8 @@ typedef enum {
   QF_OP_LINEAR_FWD = 1,
   QF_OP_LINEAR_BWD = 2,
   QF_OP_GROUPED_FWD = 3,
-  QF_OP_GROUPED_BWD = 4
+  QF_OP_GROUPED_BWD = 4,
+  QF_OP_QDQ_BATCHED = 5
 } qf_op_t;
 
 /* flags */
@@ -96,7 +97,7 @@ int qf_version(void);
 
 /* Bytes of caller-provided scratch a call needs (always a multiple of 256, never 0).
  * op = QF_OP_QDQ: M = rows, K = cols, N ignored. Linear ops: M, N, K as in the call; for grouped ops
- * M = rows_padded and `groups` = number of experts. */
+ * M = rows_padded and `groups` = number of experts. QF_OP_QDQ_BATCHED: `groups` = number of tensors, M, N, K ignored. */
 size_t qf_workspace_bytes(qf_op_t op, int64_t M, int64_t N, int64_t K, int groups);
 
 /* Reads the 4-byte status word at the start of a workspace (synchronises `stream` first).
@@ -123,6 +124,26 @@ qf_status_t qf_read_status(const void* workspace, void* stream, int* host_status
 qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, void* out_bf16,
                    void* codes, void* scales, float* tensor_scale, uint32_t flags, void* workspace,
                    size_t workspace_bytes, void* stream);
+
+/* qf_qdq for many tensors in one call. A quantization-aware training step quantizes every linear weight of the
+ * model (and ships the low-precision payload to the rollout engine, Section 3.4 "Low-precision weight
+ * synchronization"); most of those tensors are small enough that a call per tensor is launch-latency bound, and
+ * NVFP4 (Eq. nvfp4) needs each tensor's maximum before any of its blocks can be scaled. Results are exactly those
+ * of calling qf_qdq on every tensor by itself.
+ *   n            number of tensors (n = 0 is a no-op)
+ *   in, rows, cols   HOST arrays of n device pointers (BF16 [rows[i], cols[i]]) and their shapes
+ *   out_bf16, codes, scales   HOST arrays of n device pointers, layouts as in qf_qdq. Each array may be NULL as a
+ *                whole (that output is skipped for every tensor) and entry by entry; every non-empty tensor needs
+ *                at least one output. out_bf16[i] may equal in[i].
+ *   tensor_scales   NVFP4 only: DEVICE float[n], one tensor scale per tensor: written (derived from each tensor's
+ *                maximum), read with QF_TENSOR_SCALE_GIVEN, or guesses on entry and derived values on return with
+ *                QF_TENSOR_SCALE_SPECULATIVE (see that flag; a tensor quantized in place is derived directly).
+ *   workspace    qf_workspace_bytes(QF_OP_QDQ_BATCHED, 0, 0, 0, n) bytes (needed for NVFP4 without given scales)
+ * The host arrays are read during the call only. Errors as for qf_qdq, checked for every tensor before anything
+ * is enqueued. */
+qf_status_t qf_qdq_batched(qf_format_t fmt, int n, const void* const* in, const int64_t* rows, const int64_t* cols,
+                           void* const* out_bf16, void* const* codes, void* const* scales, float* tensor_scales,
+                           uint32_t flags, void* workspace, size_t workspace_bytes, void* stream);
 
 /* LoRA-QAD weight path (Eq. qad-lora, Eq. export-lora): quantize-dequantize the MERGED weight
  *     W_hat = Q^-1(Q(W + lora_scale * B A)),

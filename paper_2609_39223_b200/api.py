@@ -14,7 +14,7 @@ import torch
 
 FMT_NONE, FMT_NVFP4, FMT_MXFP4, FMT_Q4_K = 0, 1, 2, 3
 DT_BF16, DT_F32 = 0, 1
-OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD = 0, 1, 2, 3, 4
+OP_QDQ, OP_LINEAR_FWD, OP_LINEAR_BWD, OP_GROUPED_FWD, OP_GROUPED_BWD, OP_QDQ_BATCHED = 0, 1, 2, 3, 4, 5
 TENSOR_SCALE_GIVEN = 0x1
 W_TSCALE_GIVEN, A_TSCALE_GIVEN, ACCUMULATE_DW, FUSED_QDQ, AMAX_RUNNING = 0x1, 0x2, 0x4, 0x8, 0x10
 REUSE_W_HAT, REUSE_X_HAT = 0x20, 0x40
@@ -30,7 +30,7 @@ EXPORTS = [
     "qf_status_string", "qf_version", "qf_workspace_bytes", "qf_read_status", "qf_qdq", "qf_dequant", "qf_amax",
     "qf_fq_linear_fwd", "qf_fq_linear_bwd", "qf_fq_grouped_linear_fwd", "qf_fq_grouped_linear_bwd", "qf_selftest_cvt",
     "qf_selftest_div", "qf_fq_linear_fwd_noalloc", "qf_selftest_mxfp4_bf16", "qf_selftest_timeout", "qf_pack_bytes", "qf_pack", "qf_unpack", "qf_nvfp4_tensor_scale", "qf_qdq_lora",
-    "qf_fp4_matmul_native",
+    "qf_fp4_matmul_native", "qf_qdq_batched",
 ]
 NOALLOC_SCRATCH_BYTES = 32 << 20
 LAYOUT_GGUF_Q4_K, LAYOUT_FP4_SWIZZLED_SCALES = 1, 2
@@ -62,6 +62,9 @@ def lib() -> ctypes.CDLL:
         L.qf_qdq.restype = c_int
         L.qf_qdq.argtypes = [c_int, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_uint32,
                              c_void_p, c_size_t, c_void_p]
+        L.qf_qdq_batched.restype = c_int
+        L.qf_qdq_batched.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_uint32,
+                                     c_void_p, c_size_t, c_void_p]
         L.qf_dequant.restype = c_int
         L.qf_dequant.argtypes = [c_int, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p]
         L.qf_amax.restype = c_int
@@ -187,6 +190,38 @@ def qf_qdq(fmt: int, x: torch.Tensor, *, want_out=True, want_codes=True, want_sc
     _check(lib().qf_qdq(fmt, _ptr(x), rows, cols, _ptr(out), _ptr(codes), _ptr(scales), _ptr(ts), flags, _ptr(ws),
                         ws.numel(), _stream()), "qf_qdq")
     return {"out": out, "codes": codes, "scales": scales, "tensor_scale": ts}
+
+
+class QdqBatch:
+    """Marshalled argument arrays of a batched call (built once, reusable call after call: the tensors it was built
+    from must stay alive). ``out`` / ``codes`` / ``scales`` are lists of tensors; ``tensor_scales`` is a float32
+    CUDA tensor with one entry per input (NVFP4)."""
+
+    def __init__(self, fmt: int, xs, *, want_out=True, want_codes=True, want_scales=True, tensor_scales=None, ws=None):
+        self.fmt, self.xs = fmt, [_bf16(x, "x") for x in xs]
+        n = self.n = len(self.xs)
+        dev = self.xs[0].device if n else "cuda"
+        self.out = [torch.empty_like(x) for x in self.xs] if want_out else None
+        self.codes = [torch.empty((x.shape[0], x.shape[1] // 2), dtype=torch.uint8, device=dev) for x in self.xs] if want_codes else None
+        self.scales = [torch.empty(scales_shape(fmt, *x.shape), dtype=torch.uint8, device=dev) for x in self.xs] if want_scales else None
+        self.tensor_scales = tensor_scales
+        if fmt == FMT_NVFP4 and tensor_scales is None:
+            self.tensor_scales = torch.zeros(max(n, 1), dtype=torch.float32, device=dev)
+        self.ws = ws if ws is not None else workspace(OP_QDQ_BATCHED, 0, 0, 0, n, device=dev)
+        arr = lambda ts: None if ts is None else (c_void_p * max(n, 1))(*[t.data_ptr() for t in ts])
+        self._in, self._out, self._codes, self._scales = arr(self.xs), arr(self.out), arr(self.codes), arr(self.scales)
+        self._rows = (c_int64 * max(n, 1))(*[x.shape[0] for x in self.xs])
+        self._cols = (c_int64 * max(n, 1))(*[x.shape[1] for x in self.xs])
+
+    def run(self, flags: int = 0):
+        _check(lib().qf_qdq_batched(self.fmt, self.n, self._in, self._rows, self._cols, self._out, self._codes, self._scales,
+                                    _ptr(self.tensor_scales), flags, _ptr(self.ws), self.ws.numel(), _stream()), "qf_qdq_batched")
+        return self
+
+
+def qf_qdq_batched(fmt: int, xs, *, flags: int = 0, **kw) -> QdqBatch:
+    """qf_qdq over a list of tensors in one call; returns the QdqBatch holding the outputs."""
+    return QdqBatch(fmt, xs, **kw).run(flags)
 
 
 def qf_dequant(fmt: int, codes: torch.Tensor, scales: torch.Tensor, tensor_scale, rows: int, cols: int) -> torch.Tensor:

@@ -269,6 +269,7 @@ size_t qf_workspace_bytes(qf_op_t op, int64_t M, int64_t N, int64_t K, int group
   if (N < 0) N = 0;
   if (K < 0) K = 0;
   if (op == QF_OP_QDQ) return kWsHeader;
+  if (op == QF_OP_QDQ_BATCHED) return kWsHeader + round256(8 * static_cast<size_t>(groups > 0 ? groups : 0));
   const int64_t g = (op == QF_OP_GROUPED_FWD || op == QF_OP_GROUPED_BWD) ? (groups > 0 ? groups : 1) : 1;
   return linear_ws_bytes(M, N, K, g);
 }
@@ -322,6 +323,51 @@ qf_status_t qf_qdq(qf_format_t fmt, const void* in, int64_t rows, int64_t cols, 
     }
   }
   return cu(launch_qdq(q, st));
+}
+
+qf_status_t qf_qdq_batched(qf_format_t fmt, int n, const void* const* in, const int64_t* rows, const int64_t* cols,
+                           void* const* out_bf16, void* const* codes, void* const* scales, float* tensor_scales, uint32_t flags,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  if (!valid_fmt(fmt, false)) return QF_ERR_FORMAT;
+  if (n < 0) return QF_ERR_SHAPE;
+  if (n == 0) return QF_OK;
+  if (!in || !rows || !cols) return QF_ERR_NULL;
+  if (fmt == QF_FMT_NVFP4 && !tensor_scales) return QF_ERR_NULL;
+  bool in_place = false;
+  for (int i = 0; i < n; ++i) {
+    if (rows[i] < 0 || cols[i] < 0 || cols[i] % block_of(fmt)) return QF_ERR_SHAPE;
+    const bool empty = rows[i] == 0 || cols[i] == 0;
+    void* o = out_bf16 ? out_bf16[i] : nullptr;
+    void* c = codes ? codes[i] : nullptr;
+    void* sc = scales ? scales[i] : nullptr;
+    if (!empty && (!in[i] || (!o && !c && !sc))) return QF_ERR_NULL;
+    if (!aligned16(in[i]) || !aligned16(o) || !aligned16(c) || !aligned16(sc)) return QF_ERR_ALIGN;
+    if (!empty && o == in[i]) in_place = true;
+  }
+  const bool given = fmt == QF_FMT_NVFP4 && (flags & QF_TENSOR_SCALE_GIVEN);
+  const bool need_ws = fmt == QF_FMT_NVFP4 && !given;
+  const size_t ws_need = kWsHeader + round256(8 * static_cast<size_t>(n));
+  if (need_ws) {
+    if (!workspace || workspace_bytes < ws_need) return QF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return QF_ERR_ALIGN;
+  }
+  if (qf_status_t s = check_arch()) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  QdqBatchArgs a{};
+  a.fmt = fmt;
+  a.n = n;
+  a.in = in; a.rows = rows; a.cols = cols;
+  a.out = out_bf16; a.codes = codes; a.scales = scales;
+  a.tscales = tensor_scales;
+  a.given = given;
+  // a first pass with a guessed scale would overwrite an input that the second pass may still need
+  a.speculative = need_ws && (flags & QF_TENSOR_SCALE_SPECULATIVE) && !in_place;
+  a.noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
+  if (need_ws) {
+    if (cudaError_t e = cudaMemsetAsync(workspace, 0, ws_need, st)) return cu(e);
+    a.ws_words = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(workspace) + kWsHeader);
+  }
+  return cu(launch_qdq_batched(a, st));
 }
 
 qf_status_t qf_qdq_lora(qf_format_t fmt, const void* W, const void* B, const void* A, int rank, float lora_scale, int64_t rows,

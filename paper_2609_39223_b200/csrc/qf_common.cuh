@@ -149,6 +149,22 @@ struct QdqArgs {
   float lora_scale;
 };
 
+// Many tensors in one call (host arrays of device pointers and shapes); see launch_qdq_batched in qf_qdq.cu.
+struct QdqBatchArgs {
+  int fmt;
+  int n;
+  const void* const* in;
+  const int64_t* rows;
+  const int64_t* cols;
+  void* const* out;              // each array nullable as a whole, and entry by entry
+  void* const* codes;
+  void* const* scales;
+  float* tscales;                // NVFP4: device float[n], read (given / guesses) or written (derived)
+  bool given, speculative, noclip;
+  uint32_t* ws_words;            // NVFP4 without given scales: device uint32[2n], zeroed on the stream beforehand
+};
+cudaError_t launch_qdq_batched(const QdqBatchArgs& a, cudaStream_t st);
+
 cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStream_t st);
 cudaError_t launch_qdq_nvfp4_speculative(const QdqArgs& a, uint32_t* header, int amax_word, int guess_word, cudaStream_t st);
 cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStream_t st);

@@ -239,42 +239,30 @@ __device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax
 
 constexpr int kUnitsPerThread = 2;
 
+// NVFP4 per-tensor constants derived from the tensor scale: the divisor 6 * s_t of the block-scale quotient and its
+// exactly rounded reciprocal (when the divisor lies in the range where the reciprocal-based division is exact).
+struct Nvfp4Tensor {
+  float s_t, denom, rc_denom;
+  bool denom_safe;
+};
+__device__ __forceinline__ Nvfp4Tensor nvfp4_tensor(float s_t) {
+  Nvfp4Tensor t;
+  t.s_t = s_t;
+  t.denom = __fmul_rn(6.0f, s_t);
+  t.denom_safe = div_safe(t.denom);
+  t.rc_denom = t.denom_safe ? __frcp_rn(t.denom) : 0.0f;
+  return t;
+}
+
+// The grid-stride loop shared by the single-tensor and the batched FP4 kernels: this thread's units are
+// first, first + stride, ... (two in flight per iteration). Every thread of the block must call it (the optional
+// maximum reduction at the end synchronises the block).
 template <int FMT, typename Loader>
-__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t nunits,
-                                                           uint4* __restrict__ out, uint2* __restrict__ codes,
-                                                           uint8_t* __restrict__ scales,
-                                                           const float* __restrict__ tscale_in,
-                                                           const uint32_t* __restrict__ amax_bits,
-                                                           float* __restrict__ tscale_out, int opts, Nvfp4Speculation spec) {
-  const bool reverse = (opts & 1) != 0;       // walk back to front
-  const bool noclip = (opts & 2) != 0;        // MXFP4 scale rule without saturation
-  // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
-  const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
-  const Loader in = src.slice(2 * goff);
-  {
-    if (out) out += 2 * goff;
-    if (codes) codes += goff;
-    if (scales) scales += FMT == QF_FMT_NVFP4 ? goff : goff / 2;
-  }
-  float s_t = 1.0f, denom = 6.0f, rc_denom = 0.0f;
-  bool denom_safe = false;
-  if (FMT == QF_FMT_NVFP4) {
-    if (amax_bits) {
-      const float amax_t = __uint_as_float(amax_bits[blockIdx.y]);
-      s_t = amax_t == 0.0f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);            // 2688 = 6 * 448
-      // the first pass already quantized with exactly this scale: nothing to redo (every CTA decides alike)
-      if (spec.skip_guess && __float_as_uint(s_t) == *spec.skip_guess) return;
-      if (tscale_out && blockIdx.x == 0 && threadIdx.x == 0) tscale_out[blockIdx.y] = s_t;
-    } else {
-      s_t = tscale_in[blockIdx.y];
-      if (spec.guess_out && blockIdx.x == 0 && threadIdx.x == 0) *spec.guess_out = __float_as_uint(s_t);
-    }
-    denom = __fmul_rn(6.0f, s_t);
-    denom_safe = div_safe(denom);
-    rc_denom = denom_safe ? __frcp_rn(denom) : 0.0f;
-  }
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
-  const int64_t first = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+__device__ __forceinline__ void qdq_fp4_body(const Loader& in, int64_t nunits, uint4* __restrict__ out, uint2* __restrict__ codes,
+                                             uint8_t* __restrict__ scales, const Nvfp4Tensor nt, bool reverse, bool noclip,
+                                             uint32_t* __restrict__ amax_accum, int64_t first, int64_t stride) {
+  const float s_t = nt.s_t, denom = nt.denom, rc_denom = nt.rc_denom;
+  const bool denom_safe = nt.denom_safe;
   const int lane = threadIdx.x & 31;
   const int64_t warp_first = first - lane;                    // warp-uniform trip count (shuffles below)
   const int64_t nunits_up = (nunits + 31) & ~static_cast<int64_t>(31);
@@ -324,7 +312,7 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
       }
     }
   }
-  if (spec.amax_accum) {
+  if (amax_accum) {
     // the maximum of everything this pass read (padding lanes contributed zeros): for the pass that checks a
     // guessed tensor scale, or for a caller that wants max|x| reported without a separate read
     seen = __reduce_max_sync(0xFFFFFFFFu, seen);
@@ -335,9 +323,128 @@ __global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t n
       uint32_t m = 0;
 #pragma unroll
       for (int k = 0; k < kThreads / 32; ++k) m = max(m, warp_seen[k]);
-      if (m) atomicMax(spec.amax_accum, m << 16);             // BF16 bits -> FP32 bits
+      if (m) atomicMax(amax_accum, m << 16);             // BF16 bits -> FP32 bits
     }
   }
+}
+
+// The NVFP4 tensor scale a block works with, from whichever source the call uses: `amax_bits` (derive it; the scale is
+// also stored to *tscale_out by the slice's first thread) or `tscale_in` (supplied, or a guess in the speculative
+// first pass, whose bits are then recorded in *guess_out). Returns false when the block has nothing to do: the
+// speculative second pass found the derived scale equal to the guess the first pass quantized with.
+__device__ __forceinline__ bool nvfp4_resolve_scale(const float* tscale_in, const uint32_t* amax_bits, float* tscale_out,
+                                                    uint32_t* guess_out, const uint32_t* skip_guess, float& s_t) {
+  if (amax_bits) {
+    const float amax_t = __uint_as_float(*amax_bits);
+    s_t = amax_t == 0.0f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);            // 2688 = 6 * 448
+    // the first pass already quantized with exactly this scale: nothing to redo (every CTA decides alike)
+    if (skip_guess && __float_as_uint(s_t) == *skip_guess) return false;
+    if (tscale_out && blockIdx.x == 0 && threadIdx.x == 0) *tscale_out = s_t;
+  } else {
+    s_t = *tscale_in;
+    if (guess_out && blockIdx.x == 0 && threadIdx.x == 0) *guess_out = __float_as_uint(s_t);
+  }
+  return true;
+}
+
+template <int FMT, typename Loader>
+__global__ void __launch_bounds__(kThreads) qdq_fp4_kernel(Loader src, int64_t nunits,
+                                                           uint4* __restrict__ out, uint2* __restrict__ codes,
+                                                           uint8_t* __restrict__ scales,
+                                                           const float* __restrict__ tscale_in,
+                                                           const uint32_t* __restrict__ amax_bits,
+                                                           float* __restrict__ tscale_out, int opts, Nvfp4Speculation spec) {
+  const bool reverse = (opts & 1) != 0;       // walk back to front
+  const bool noclip = (opts & 2) != 0;        // MXFP4 scale rule without saturation
+  // gridDim.y > 1: one tensor of nunits units per y-slice, each with its own tensor scale (NVFP4 experts)
+  const int64_t goff = static_cast<int64_t>(blockIdx.y) * nunits;
+  const Loader in = src.slice(2 * goff);
+  {
+    if (out) out += 2 * goff;
+    if (codes) codes += goff;
+    if (scales) scales += FMT == QF_FMT_NVFP4 ? goff : goff / 2;
+  }
+  float s_t = 1.0f;
+  if (FMT == QF_FMT_NVFP4) {
+    if (!nvfp4_resolve_scale(tscale_in ? tscale_in + blockIdx.y : nullptr, amax_bits ? amax_bits + blockIdx.y : nullptr,
+                             tscale_out ? tscale_out + blockIdx.y : nullptr, spec.guess_out, spec.skip_guess, s_t))
+      return;
+  }
+  qdq_fp4_body<FMT, Loader>(in, nunits, out, codes, scales, nvfp4_tensor(s_t), reverse, noclip, spec.amax_accum,
+                            static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x, static_cast<int64_t>(gridDim.x) * kThreads);
+}
+
+// ---- batched form: many tensors, each with its own pointers and size, in one launch -----------------------
+// The table travels as a kernel parameter (no device-side table to allocate or copy). blockIdx.y selects the tensor;
+// blocks beyond a short tensor's need leave at once.
+constexpr int kMaxBatch = 64;
+struct QdqBatch {
+  const uint4* in[kMaxBatch];
+  uint4* out[kMaxBatch];
+  void* codes[kMaxBatch];
+  void* scales[kMaxBatch];
+  int64_t nunits[kMaxBatch];       // FP4: 16-element units; Q4_K: 32-weight sub-blocks
+};
+
+// role split of one launch: y-slices [0, n_qdq) quantize tensors of `q`, y-slices [n_qdq, n_qdq + n_amax) take the
+// absolute maximum of the tensors of `a` (the NEXT sub-batch): its reads overlap the writes of this one and leave those
+// tensors in L2 for the launch that quantizes them.
+struct AmaxBatch {
+  const uint4* in[kMaxBatch];
+  int64_t nchunks[kMaxBatch];
+};
+
+__device__ __forceinline__ void amax_block(const uint4* __restrict__ in, int64_t nchunks, uint32_t* __restrict__ amax_bits,
+                                           int64_t first, int64_t stride) {
+  uint32_t m = 0;
+  int64_t i = first;
+  for (; i + 3 * stride < nchunks; i += 4 * stride) {
+    const uint4 a = __ldg(in + i), b = __ldg(in + i + stride), c = __ldg(in + i + 2 * stride), d = __ldg(in + i + 3 * stride);
+    m = max(m, max(max(chunk_amax_bits(a), chunk_amax_bits(b)), max(chunk_amax_bits(c), chunk_amax_bits(d))));
+  }
+  for (; i < nchunks; i += stride) m = max(m, chunk_amax_bits(__ldg(in + i)));
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  __shared__ uint32_t warp_max[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if (threadIdx.x == 0 && m) atomicMax(amax_bits, m << 16);     // BF16 bits -> FP32 bits
+  }
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kThreads) qdq_fp4_batched_kernel(const __grid_constant__ QdqBatch q, int n_qdq,
+                                                                   const __grid_constant__ AmaxBatch a,
+                                                                   const float* __restrict__ tscale_in,
+                                                                   const uint32_t* __restrict__ amax_bits,
+                                                                   float* __restrict__ tscale_out, int opts,
+                                                                   uint32_t* __restrict__ amax_accum, uint32_t* __restrict__ guess_out,
+                                                                   const uint32_t* __restrict__ skip_guess,
+                                                                   uint32_t* __restrict__ next_amax_bits) {
+  const int64_t first = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
+  const int t = blockIdx.y;
+  if (t >= n_qdq) {
+    const int u = t - n_qdq;
+    if (static_cast<int64_t>(blockIdx.x) * kThreads >= a.nchunks[u]) return;
+    amax_block(a.in[u], a.nchunks[u], next_amax_bits + u, first, stride);
+    return;
+  }
+  const int64_t nunits = q.nunits[t];
+  // (block-uniform; block 0 stays even for an empty tensor: it stores the tensor scale, 1.0)
+  if (blockIdx.x > 0 && static_cast<int64_t>(blockIdx.x) * kThreads >= nunits) return;
+  float s_t = 1.0f;
+  if (FMT == QF_FMT_NVFP4) {
+    if (!nvfp4_resolve_scale(tscale_in ? tscale_in + t : nullptr, amax_bits ? amax_bits + t : nullptr,
+                             tscale_out ? tscale_out + t : nullptr, guess_out ? guess_out + t : nullptr,
+                             skip_guess ? skip_guess + t : nullptr, s_t))
+      return;
+  }
+  qdq_fp4_body<FMT, PlainLoader>(PlainLoader{q.in[t]}, nunits, q.out[t], static_cast<uint2*>(q.codes[t]),
+                                 static_cast<uint8_t*>(q.scales[t]), nvfp4_tensor(s_t), (opts & 1) != 0, (opts & 2) != 0,
+                                 amax_accum ? amax_accum + t : nullptr, first, stride);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -408,13 +515,11 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
   }
 }
 
+// grid-stride loop shared by the single-tensor and the batched Q4_K kernels: sub-blocks first, first + stride, ...
 template <typename Loader>
-__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(Loader in, int64_t nsub,
-                                                           uint4* __restrict__ out, uint4* __restrict__ codes,
-                                                           uint4* __restrict__ scales) {
+__device__ __forceinline__ void qdq_q4k_body(const Loader& in, int64_t nsub, uint4* __restrict__ out, uint4* __restrict__ codes,
+                                             uint4* __restrict__ scales, int64_t first, int64_t stride) {
   const int lane = threadIdx.x & 31;
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
-  const int64_t first = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
   // nsub (sub-blocks) is a multiple of 8; a warp covers 32 of them, so the last warp may be partly idle
   for (int64_t i = first; i - lane < nsub; i += stride) {
     const bool ok = i < nsub;
@@ -481,6 +586,22 @@ __global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(Loa
       }
     }
   }
+}
+
+template <typename Loader>
+__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_kernel(Loader in, int64_t nsub,
+                                                           uint4* __restrict__ out, uint4* __restrict__ codes,
+                                                           uint4* __restrict__ scales) {
+  qdq_q4k_body<Loader>(in, nsub, out, codes, scales, static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x,
+                       static_cast<int64_t>(gridDim.x) * kThreads);
+}
+
+__global__ void __launch_bounds__(kThreads, QF_Q4K_MINBLOCKS) qdq_q4k_batched_kernel(const __grid_constant__ QdqBatch q) {
+  const int t = blockIdx.y;
+  const int64_t nsub = q.nunits[t];
+  if (static_cast<int64_t>(blockIdx.x) * kThreads >= nsub) return;
+  qdq_q4k_body<PlainLoader>(PlainLoader{q.in[t]}, nsub, q.out[t], static_cast<uint4*>(q.codes[t]), static_cast<uint4*>(q.scales[t]),
+                            static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x, static_cast<int64_t>(gridDim.x) * kThreads);
 }
 
 // exhaustive comparison of the reciprocal-based division with the IEEE divide: every x in xs against
@@ -642,6 +763,103 @@ cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStre
                                                                       static_cast<const __nv_bfloat16*>(in) + nchunks * 8, ntail,
                                                                       amax_bits);
   return cudaGetLastError();
+}
+
+// ---- batched launches --------------------------------------------------------------------------------
+// Many tensors per call (every linear weight of a model is quantized each step for weight synchronisation, Section 3.4):
+// MXFP4, Q4_K and NVFP4 with supplied scales take one launch per 64 tensors. NVFP4 with derived scales needs every
+// tensor's maximum before its blocks can be scaled; the batch is cut into sub-batches small enough to stay in L2
+// (kSubBatchBytes of input), and launch j quantizes sub-batch j-1 while its spare y-slices take the maxima of
+// sub-batch j: S + 1 launches for S sub-batches instead of three per tensor, with the second read of every tensor
+// served from L2. With speculated scales (the previous step's) one launch quantizes with the guesses and gathers the
+// true maxima, a second one derives the scales and requantizes only the tensors whose guess was wrong.
+constexpr int64_t kSubBatchBytes = 24ll << 20;
+
+static int batched_grid_x(int64_t max_items, int per_thread, int ny, int blocks_per_sm) {
+  int64_t gx = (max_items + static_cast<int64_t>(kThreads) * per_thread - 1) / (static_cast<int64_t>(kThreads) * per_thread);
+  if (blocks_per_sm > 0) {
+    const int64_t cap = (static_cast<int64_t>(kNumSMs) * blocks_per_sm + ny - 1) / ny;
+    if (gx > cap) gx = cap;
+  }
+  if (gx > 0x7FFFFFFF) gx = 0x7FFFFFFF;
+  return static_cast<int>(gx < 1 ? 1 : gx);
+}
+
+cudaError_t launch_qdq_batched(const QdqBatchArgs& a, cudaStream_t st) {
+  const int unit = a.fmt == QF_FMT_Q4_K ? 32 : 16;
+  auto fill = [&](QdqBatch& q, int t0, int cnt, int64_t& max_units) {
+    max_units = 0;
+    for (int i = 0; i < cnt; ++i) {
+      const int t = t0 + i;
+      q.in[i] = static_cast<const uint4*>(a.in[t]);
+      q.out[i] = a.out ? static_cast<uint4*>(a.out[t]) : nullptr;
+      q.codes[i] = a.codes ? a.codes[t] : nullptr;
+      q.scales[i] = a.scales ? a.scales[t] : nullptr;
+      q.nunits[i] = a.rows[t] * a.cols[t] / unit;
+      if (q.nunits[i] > max_units) max_units = q.nunits[i];
+    }
+  };
+  const int opts = a.noclip ? 2 : 0;
+  static const AmaxBatch no_amax{};
+  if (a.fmt != QF_FMT_NVFP4 || a.given || a.speculative) {
+    for (int t0 = 0; t0 < a.n; t0 += kMaxBatch) {
+      const int cnt = a.n - t0 < kMaxBatch ? a.n - t0 : kMaxBatch;
+      QdqBatch q{};
+      int64_t mx;
+      fill(q, t0, cnt, mx);
+      if (a.fmt == QF_FMT_Q4_K) {
+        qdq_q4k_batched_kernel<<<dim3(batched_grid_x(mx, 1, cnt, 32), cnt), kThreads, 0, st>>>(q);
+      } else if (a.fmt == QF_FMT_MXFP4) {
+        qdq_fp4_batched_kernel<QF_FMT_MXFP4><<<dim3(batched_grid_x(mx, kUnitsPerThread, cnt, 0), cnt), kThreads, 0, st>>>(
+            q, cnt, no_amax, nullptr, nullptr, nullptr, opts, nullptr, nullptr, nullptr, nullptr);
+      } else if (a.given) {
+        qdq_fp4_batched_kernel<QF_FMT_NVFP4><<<dim3(batched_grid_x(mx, kUnitsPerThread, cnt, 16), cnt), kThreads, 0, st>>>(
+            q, cnt, no_amax, a.tscales + t0, nullptr, nullptr, 0, nullptr, nullptr, nullptr, nullptr);
+      } else {
+        uint32_t* amax = a.ws_words + t0;
+        uint32_t* guess = a.ws_words + a.n + t0;
+        const dim3 grid(batched_grid_x(mx, kUnitsPerThread, cnt, 16), cnt);
+        qdq_fp4_batched_kernel<QF_FMT_NVFP4><<<grid, kThreads, 0, st>>>(q, cnt, no_amax, a.tscales + t0, nullptr, nullptr, 0, amax,
+                                                                        guess, nullptr, nullptr);
+        if (cudaError_t e = cudaGetLastError()) return e;
+        qdq_fp4_batched_kernel<QF_FMT_NVFP4><<<grid, kThreads, 0, st>>>(q, cnt, no_amax, nullptr, amax, a.tscales + t0, 0, nullptr,
+                                                                        nullptr, guess, nullptr);
+      }
+      if (cudaError_t e = cudaGetLastError()) return e;
+    }
+    return cudaSuccess;
+  }
+  // NVFP4, derived scales: software pipeline over L2-sized sub-batches
+  int prev0 = 0, prev_cnt = 0;             // the sub-batch whose maxima are already being gathered / are complete
+  int t = 0;
+  while (t < a.n || prev_cnt > 0) {
+    int cnt = 0;
+    int64_t bytes = 0;
+    while (t + cnt < a.n && cnt < kMaxBatch) {
+      const int64_t b = a.rows[t + cnt] * a.cols[t + cnt] * 2;
+      if (cnt > 0 && bytes + b > kSubBatchBytes) break;
+      bytes += b;
+      ++cnt;
+    }
+    QdqBatch q{};
+    AmaxBatch am{};
+    int64_t mq = 0, ma = 0;
+    if (prev_cnt > 0) fill(q, prev0, prev_cnt, mq);
+    for (int i = 0; i < cnt; ++i) {
+      am.in[i] = static_cast<const uint4*>(a.in[t + i]);
+      am.nchunks[i] = a.rows[t + i] * a.cols[t + i] / 8;
+      if (am.nchunks[i] > ma) ma = am.nchunks[i];
+    }
+    const int ny = prev_cnt + cnt;
+    const int64_t gq = batched_grid_x(mq, kUnitsPerThread, ny, 16), ga = batched_grid_x(ma, 4, ny, 16);
+    qdq_fp4_batched_kernel<QF_FMT_NVFP4><<<dim3(static_cast<unsigned>(gq > ga ? gq : ga), ny), kThreads, 0, st>>>(
+        q, prev_cnt, am, nullptr, a.ws_words + prev0, a.tscales + prev0, 0, nullptr, nullptr, nullptr, a.ws_words + t);
+    if (cudaError_t e = cudaGetLastError()) return e;
+    prev0 = t;
+    prev_cnt = cnt;
+    t += cnt;
+  }
+  return cudaSuccess;
 }
 
 static LoraLoader lora_loader(const QdqArgs& a) {

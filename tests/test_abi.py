@@ -109,6 +109,22 @@ def test_linear_argument_errors_need_no_gpu():
     assert g(P, P, P, 0, P, 4, 512, N, K, api.FMT_NVFP4, 0, None, None, 0, P, 1 << 30, None) == 1
 
 
+def test_batched_argument_errors_need_no_gpu():
+    L = api.lib()
+    arr = lambda *v: (api.c_void_p * len(v))(*v)
+    i64 = lambda *v: (api.c_int64 * len(v))(*v)
+    call = lambda fmt, n, ins, rows, cols, outs, ts, ws, wsb: L.qf_qdq_batched(fmt, n, ins, rows, cols, outs, None, None, ts, 0, ws, wsb, None)
+    assert call(api.FMT_MXFP4, -1, arr(P), i64(4), i64(64), arr(P), None, None, 0) == 2
+    assert call(api.FMT_MXFP4, 0, None, None, None, None, None, None, 0) == 0
+    assert call(api.FMT_MXFP4, 1, None, i64(4), i64(64), arr(P), None, None, 0) == 1
+    assert call(api.FMT_MXFP4, 2, arr(P, P), i64(4, 4), i64(64, 48), arr(P, P), None, None, 0) == 2          # second tensor: bad cols
+    assert call(api.FMT_MXFP4, 2, arr(P, P + 4), i64(4, 4), i64(64, 64), arr(P, P), None, None, 0) == 3      # second tensor: misaligned
+    assert call(api.FMT_MXFP4, 1, arr(P), i64(4), i64(64), None, None, None, 0) == 1                          # no output at all
+    assert call(api.FMT_NVFP4, 1, arr(P), i64(4), i64(64), arr(P), None, P, 1 << 20) == 1                     # NVFP4 needs the scale array
+    assert call(api.FMT_NVFP4, 3, arr(P, P, P), i64(4, 4, 4), i64(64, 64, 64), arr(P, P, P), P, P, 256) == 5  # workspace too small
+    assert api.qf_workspace_bytes(api.OP_QDQ_BATCHED, 0, 0, 0, 3) == 512
+
+
 def test_calls_fail_loudly_without_a_device():
     import torch
     if torch.cuda.is_available():
