@@ -8,7 +8,12 @@ MXFP4 weights and activations, forward plus straight-through backward (dX and dW
 X [8192,4096], W [12288,4096], dY [8192,12288] — i.e. two quantize-dequantize passes over W and X
 (forward, and again in the backward, since the fake-quantized copies are transient) and three BF16
 tensor-core matmuls. Prints ONE JSON line (rank 0). Multi-GPU runs are independent replicas of
-the same workload (the path has no exchange step): weak scaling, no data-path collective.
+the same workload (the path has no exchange step): weak scaling, no data-path collective. With
+``--gpus N`` (N > 1) and no torchrun environment the script starts the N ranks itself.
+
+Beside the headline the line carries: the matmul's roofline record (with the SM clock the kernel itself
+measured), a sustained run of at least two seconds, the quantizer bandwidths, the end-to-end figure with host
+buffers, the CPU oracle's rate, and the other named workloads (``other_workloads``).
 
 `--impl reference` times the CPU oracle (the only other place this file may execute `oracle/`).
 """
@@ -17,6 +22,9 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -29,7 +37,10 @@ M, N, K = 8192, 12288, 4096
 WORKLOAD = "mxfp4_w4a4_linear_fwd_bwd_8192x4096x12288"
 FLOP_PER_GEMM = 2.0 * M * N * K
 FLOP_PER_STEP = 3.0 * FLOP_PER_GEMM
-SECTIONS = ("roofline", "qdq", "e2e", "cpu")
+SECTIONS = ("roofline", "sustained", "qdq", "e2e", "cpu", "configs")
+DATASHEET_TFLOPS = 2250.0            # dense BF16, nominal
+TENSOR_FLOP_PER_CLK_PER_SM = 8192    # dense BF16 multiply-adds x 2 per SM per clock (2250e12 / 148 / 1.86e9)
+NUM_SMS = 148
 
 
 def _set_shape(spec: str):
@@ -51,8 +62,22 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
 
 
+def _profiled_traffic(m: int, n: int, k: int):
+    """Mean DRAM bytes per matmul launch of a step, as the committed ncu summary of that shape records it
+    (a line ``traffic_bytes_per_launch M=.. N=.. K=..: <bytes>``); None when no capture of this shape is on file."""
+    p = ROOT / "profiles" / "gemm_pair_kernel_mxfp4_linear.md"
+    if not p.exists():
+        return None
+    pat = re.compile(r"traffic_bytes_per_launch\s+M=(\d+)\s+N=(\d+)\s+K=(\d+):\s*([0-9.eE+]+)")
+    for mm in pat.finditer(p.read_text()):
+        if (int(mm.group(1)), int(mm.group(2)), int(mm.group(3))) == (m, n, k):
+            return float(mm.group(4))
+    return None
+
+
 class ClockSampler:
-    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read-only)."""
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read-only), about once
+    per millisecond."""
 
     def __init__(self, index: int):
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -83,7 +108,7 @@ class ClockSampler:
                         self.reasons.add(n)
             except Exception:
                 pass
-            time.sleep(0.005)
+            time.sleep(0.001)
 
     def __enter__(self):
         if self.nv:
@@ -98,8 +123,8 @@ class ClockSampler:
 
     def summary(self):
         s = sorted(self.samples)
-        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(s)}
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_min_mhz": s[0] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
 
 
 def _physical_gpu_index(local_rank: int) -> int:
@@ -110,6 +135,42 @@ def _physical_gpu_index(local_rank: int) -> int:
         except Exception:
             return local_rank
     return local_rank
+
+
+# -------------------------------------------------------------------------------------------------
+# launcher: --gpus N without a torchrun environment starts N ranks
+# -------------------------------------------------------------------------------------------------
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv: list[str]) -> int:
+    """Re-runs this script as n ranks under torch.distributed.run (one process per GPU, rendezvous on 127.0.0.1)
+    and returns its exit code. Rank 0 of the children prints the JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(_free_port()), str(Path(__file__).resolve()), *argv]
+    return subprocess.call(cmd)
+
+
+def run_dry(args):
+    """The launch and timing protocol alone, with no GPU: ranks rendezvous over gloo, "run" steps that only sleep,
+    take the max time over ranks and print the line. What the CPU tests use to check `--gpus N`."""
+    from paper_2609_39223_b200 import replicas
+    world, rank, _ = replicas.world()
+    replicas.init("gloo")
+    replicas.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.002 * (1 + rank))
+    ms = replicas.max_over_ranks((time.perf_counter() - t0) * 1e3)
+    replicas.barrier()
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "impl": args.impl, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": ms / max(1, args.steps), "scaling": "weak"}))
+    replicas.finish()
 
 
 # -------------------------------------------------------------------------------------------------
@@ -136,6 +197,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     import oracle
     cores = oracle.num_threads()
     n_rows = 512
@@ -155,7 +217,7 @@ def run_reference(args):
     sample = f"fwd+dX+dW on a [{m_rows},{K}] x [{n_rows},{K}] slice per step (QDQ of both slices included)"
     print(json.dumps({
         "impl": "reference", "metric": "fake-quant linear fwd+bwd TFLOPS", "value": value, "unit": "TFLOP/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(1, args.steps),
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "sample": sample},
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -165,7 +227,7 @@ def run_reference(args):
 
 
 # -------------------------------------------------------------------------------------------------
-# the other named workloads (parity-test cases; measured on request with --sections ...,configs)
+# the other named workloads
 # -------------------------------------------------------------------------------------------------
 
 def _time_ms(torch, fn, reps=5, warm=3):
@@ -181,45 +243,78 @@ def _time_ms(torch, fn, reps=5, warm=3):
     return a.elapsed_time(b) / reps
 
 
-def measure_other_workloads(torch, api, synth, dev, peaks):
+def _timed_region(torch, gpu_index, fn, min_seconds=1.0, warm=3, probe=3):
+    """ms per call of fn over a region of at least min_seconds, with the clocks sampled during that region."""
+    est = _time_ms(torch, fn, reps=probe, warm=warm)
+    reps = max(probe, int(min_seconds * 1e3 / max(est, 1e-3)) + 1)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    with ClockSampler(gpu_index) as clk:
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps, reps, clk.summary()
+
+
+def _graph(torch, fn):
+    fn(); torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()          # replayed as a graph: the Python binding's per-call cost is not GPU time
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
     out = {}
-    # 1: NVFP4 QDQ of 2048x2048 weights, a rotating set of 32 matrices (268 MB, more than twice L2)
+    hbm = peaks["hbm_gbs"]
+    rate = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
+    bw = lambda g: {"gbs": g, "frac_of_measured_hbm": g / hbm, "frac_of_8000_nominal": g / 8000.0}
+    # ---- 1: NVFP4 QDQ of 2048x2048 weights (all outputs, scale derived from the tensor) -----------------
     mats = [synth.weight_with_outliers(2048, 2048, seed=i, device=dev) for i in range(32)]
     o = torch.empty_like(mats[0]); c = torch.empty((2048, 1024), dtype=torch.uint8, device=dev)
     sc = torch.empty((2048, 128), dtype=torch.uint8, device=dev); wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
     ts1 = torch.empty(1, dtype=torch.float32, device=dev)
-    run1 = lambda: [api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq, tensor_scale=None, ts_out=ts1) for m in mats]
-    run1(); torch.cuda.synchronize()
-    g1 = torch.cuda.CUDAGraph()                  # replayed as a graph: the Python binding's per-call cost is not GPU time
-    with torch.cuda.graph(g1):
-        run1()
-    ms = _time_ms(torch, g1.replay) / 32
-    out["nvfp4_qdq_2048x2048"] = {"us_per_matrix": ms * 1e3, "gbs": 19136516 / (ms * 1e-3) / 1e9,
-                                  "note": "32 distinct matrices in rotation (cold L2), replayed as one CUDA graph; includes the header memset and the amax pre-pass"}
-    del mats
-    # 3: Q4_K QDQ over all linear weights of the 32-layer dense decoder (one layer's buffers reused 32 times)
-    layer = [synth.randn_bf16((r, cc), 0.02, 100 + i, device=dev) for i, (_, r, cc) in enumerate(synth.DENSE_DECODER_LAYER)]
-    outs = [torch.empty_like(w) for w in layer]
-    codes = [torch.empty((w.shape[0], w.shape[1] // 2), dtype=torch.uint8, device=dev) for w in layer]
-    scs = [torch.empty(api.scales_shape(api.FMT_Q4_K, *w.shape), dtype=torch.uint8, device=dev) for w in layer]
+    one = lambda m: api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq, tensor_scale=None, ts_out=ts1)
+    nbytes = 19136516
+    g_cold = _graph(torch, lambda: [one(m) for m in mats])              # 32 distinct matrices, 268 MB: more than twice L2
+    g_warm = _graph(torch, lambda: [one(mats[0]) for _ in range(32)])   # one matrix, back to back
+    batch = api.QdqBatch(api.FMT_NVFP4, mats)
+    g_batch = _graph(torch, batch.run)
+    g_spec = _graph(torch, lambda: batch.run(api.TENSOR_SCALE_SPECULATIVE))   # guesses = the scales the previous call derived
+    cfg1 = {"bytes_per_matrix": nbytes, "outputs": "codes, E4M3 block scales, FP32 tensor scale, BF16 dequantized",
+            "note": "every variant replayed as one CUDA graph of 32 matrices; single = qf_qdq per matrix (header memset + amax "
+                    "pre-pass + quantize), batched = one qf_qdq_batched call for the 32 matrices"}
+    for name, g in (("single_cold_l2", g_cold), ("single_warm_l2", g_warm), ("batched_32", g_batch),
+                    ("batched_32_speculated_scales_hit", g_spec)):
+        ms, reps, clk = _timed_region(torch, gpu_index, g.replay, min_seconds=0.2)
+        cfg1[name] = {"us_per_matrix": ms * 1e3 / 32, **bw(rate(32 * nbytes, ms)), "clocks": clk}
+    out["nvfp4_qdq_2048x2048"] = cfg1
+    del mats, batch, g_cold, g_warm, g_batch, g_spec
+    # ---- 3: Q4_K QDQ over all linear weights of the 32-layer dense decoder, per-layer seeds (14 GB of weights
+    # resident; outputs go to one layer's buffers, reused) ------------------------------------------------------
+    layers = [[synth.dense_decoder_weight(l, name, device=dev) for name, _, _ in synth.DENSE_DECODER_LAYER]
+              for l in range(synth.DENSE_DECODER_LAYERS)]
+    outs = [torch.empty_like(w) for w in layers[0]]
+    codes = [torch.empty((w.shape[0], w.shape[1] // 2), dtype=torch.uint8, device=dev) for w in layers[0]]
+    scs = [torch.empty(api.scales_shape(api.FMT_Q4_K, *w.shape), dtype=torch.uint8, device=dev) for w in layers[0]]
 
     def q4k_all():
-        for _ in range(synth.DENSE_DECODER_LAYERS):
+        for layer in layers:
             for w, oo, cc, ss in zip(layer, outs, codes, scs):
                 api.qf_qdq(api.FMT_Q4_K, w, out=oo, codes=cc, scales=ss, ws=wsq)
-    q4k_all(); torch.cuda.synchronize()
-    g3 = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g3):
-        q4k_all()
-    ms = _time_ms(torch, g3.replay, reps=3, warm=1)
+    g3 = _graph(torch, q4k_all)
+    ms, reps, clk = _timed_region(torch, gpu_index, g3.replay, min_seconds=0.5, warm=1, probe=2)
     elems = synth.dense_decoder_layer_elems() * synth.DENSE_DECODER_LAYERS
-    out["q4k_qdq_dense_decoder_32_layers"] = {"ms": ms, "elements": elems, "gbs": elems * 4.5625 / (ms * 1e-3) / 1e9,
-                                              "frac_of_measured_hbm": elems * 4.5625 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    del layer, outs, codes, scs
-    # 4: NVFP4 weight-only linear, one 32K-token sequence, up and down projections, fwd + bwd
+    out["q4k_qdq_dense_decoder_32_layers"] = {"ms": ms, "elements": elems, **bw(rate(elems * 4.5625, ms)), "reps": reps, "clocks": clk,
+                                              "note": "224 distinct weight tensors (per-layer seeds), one qf_qdq call each, as one CUDA graph"}
+    del layers, outs, codes, scs, g3
+    torch.cuda.empty_cache()
+    # ---- 4: NVFP4 weight-only linear, one 32K-token sequence, up and down projections, fwd + bwd ---------------
     Mt = 32768
-    tot_ms, tot_fl = 0.0, 0.0
-    for (Nn, Kk) in ((14336, 4096), (4096, 14336)):
+    tot_ms, tot_fl, parts = 0.0, 0.0, {}
+    for pname, (Nn, Kk) in (("up", (14336, 4096)), ("down", (4096, 14336))):
         cse = synth.linear_case(Mt, Nn, Kk, seed=4, device=dev, outlier_channels=0)
         ws4 = api.workspace(api.OP_LINEAR_BWD, Mt, Nn, Kk, device=dev)
         Y = torch.empty((Mt, Nn), dtype=torch.bfloat16, device=dev); dX = torch.empty((Mt, Kk), dtype=torch.bfloat16, device=dev)
@@ -228,49 +323,64 @@ def measure_other_workloads(torch, api, synth, dev, peaks):
         def f4():
             api.qf_fq_linear_fwd(cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, Y=Y, w_tscale=wts)
             api.qf_fq_linear_bwd(cse.dY, cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, dX=dX, dW=dW, w_tscale=wts)
-        tot_ms += _time_ms(torch, f4, reps=3, warm=2)
-        tot_fl += 3 * 2.0 * Mt * Nn * Kk
+        ms, reps, clk = _timed_region(torch, gpu_index, f4, min_seconds=1.0, warm=2, probe=2)
+        fl = 3 * 2.0 * Mt * Nn * Kk
+        parts[pname] = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "reps": reps, "clocks": clk}
+        tot_ms += ms; tot_fl += fl
         del cse, ws4, Y, dX, dW
-    out["nvfp4_weight_only_linear_32k_tokens_up_down"] = {"ms": tot_ms, "tflops": tot_fl / (tot_ms * 1e-3) / 1e12,
-                                                           "frac_of_2250_datasheet": tot_fl / (tot_ms * 1e-3) / 1e12 / 2250.0}
-    # 5: MoE grouped MXFP4 W4A4: 128 experts, top-8 of 16384 tokens, gate + up + down, fwd + bwd. The gate and up
+    t4 = tot_fl / (tot_ms * 1e-3) / 1e12
+    out["nvfp4_weight_only_linear_32k_tokens_up_down"] = {"ms": tot_ms, "tflops": t4, "frac_of_2250_datasheet": t4 / DATASHEET_TFLOPS,
+                                                           "frac_of_measured_sustained": t4 / peaks["bf16_sustained"],
+                                                           "frac_of_measured_burst": t4 / peaks["bf16_burst"], **parts}
+    # ---- 5: MoE grouped MXFP4 W4A4: 128 experts, top-8 of 16384 tokens, gate + up + down, fwd + bwd. The gate and up
     # projections are stored as one [E, 2F, H] weight, as serving engines keep them: the same products (the quantizer's
     # blocks run along H, so quantizing the concatenation is concatenating the quantized halves), and the routed
-    # activations are quantized once for both.
+    # activations are quantized once for both. ------------------------------------------------------------------------
     tokens, E, top_k, H, F = 16384, 128, 8, 2048, 768
     r = synth.moe_routing(tokens, E, top_k, seed=0)
     rows = int(r.group_offsets[-1]); offs = r.group_offsets.to(dev)
     fmt = api.FMT_MXFP4
-    tot_ms, tot_reuse_ms = 0.0, 0.0
-    for (Nn, Kk, times) in ((2 * F, H, 1), (H, F, 1)):
+    res = {k: [0.0, None] for k in ("default", "reuse", "bf16_dw")}
+    for (Nn, Kk) in ((2 * F, H), (H, F)):
         Xp = synth.randn_bf16((rows, Kk), 1.0, 5, device=dev); Xp[(r.token_of_row < 0).to(dev)] = 0
         Wg = synth.randn_bf16((E, Nn, Kk), 0.02, 6, device=dev)
         dYp = synth.randn_bf16((rows, Nn), 1e-3, 7, device=dev); dYp[(r.token_of_row < 0).to(dev)] = 0
         ws5 = api.workspace(api.OP_GROUPED_BWD, rows, Nn, Kk, E, device=dev)
         Y = torch.empty((rows, Nn), dtype=torch.bfloat16, device=dev); dX = torch.empty((rows, Kk), dtype=torch.bfloat16, device=dev)
         dW = torch.empty((E, Nn, Kk), dtype=torch.float32, device=dev)
+        dW16 = torch.empty((E, Nn, Kk), dtype=torch.bfloat16, device=dev)
 
-        def f5():
+        def f5(dw=dW, flags=0):
             api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
-            api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dW)
-
-        def f5_reuse():          # the backward keeps the forward's fake-quantized copies instead of recomputing them
-            api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
-            api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dW, flags=api.REUSE_W_HAT | api.REUSE_X_HAT)
-        tot_ms += times * _time_ms(torch, f5, reps=10, warm=3)
-        tot_reuse_ms += times * _time_ms(torch, f5_reuse, reps=10, warm=3)
-        del Xp, Wg, dYp, ws5, Y, dX, dW
+            api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dw, flags=flags)
+        for key, fn in (("default", f5), ("reuse", lambda: f5(flags=api.REUSE_W_HAT | api.REUSE_X_HAT)), ("bf16_dw", lambda: f5(dw=dW16))):
+            ms, reps, clk = _timed_region(torch, gpu_index, fn, min_seconds=1.0 if key == "default" else 0.3)
+            res[key][0] += ms
+            res[key][1] = clk
+        del Xp, Wg, dYp, ws5, Y, dX, dW, dW16
     fl = 3 * 3 * 2.0 * tokens * top_k * H * F
-    out["moe_grouped_mxfp4_128_experts"] = {"ms": tot_ms, "tflops": fl / (tot_ms * 1e-3) / 1e12, "routed_rows": tokens * top_k,
-                                            "layout": "gate and up as one [128, 1536, 2048] grouped weight, down [128, 2048, 768]",
-                                            "ms_reusing_forward_copies": tot_reuse_ms, "tflops_reusing_forward_copies": fl / (tot_reuse_ms * 1e-3) / 1e12,
-                                            "padded_rows": rows, "frac_of_2250_datasheet": fl / (tot_ms * 1e-3) / 1e12 / 2250.0}
+    tf = lambda ms: fl / (ms * 1e-3) / 1e12
+    out["moe_grouped_mxfp4_128_experts"] = {
+        "ms": res["default"][0], "tflops": tf(res["default"][0]), "frac_of_2250_datasheet": tf(res["default"][0]) / DATASHEET_TFLOPS,
+        "frac_of_measured_sustained": tf(res["default"][0]) / peaks["bf16_sustained"], "clocks": res["default"][1],
+        "routed_rows": tokens * top_k, "padded_rows": rows,
+        "layout": "gate and up as one [128, 1536, 2048] grouped weight, down [128, 2048, 768]; dW in FP32",
+        "ms_reusing_forward_copies": res["reuse"][0], "tflops_reusing_forward_copies": tf(res["reuse"][0]),
+        "ms_with_bf16_dw": res["bf16_dw"][0], "tflops_with_bf16_dw": tf(res["bf16_dw"][0])}
     return out
 
 
 # -------------------------------------------------------------------------------------------------
 # our arm
 # -------------------------------------------------------------------------------------------------
+
+def _kernel_clock_mhz(ws):
+    """SM clock the last matmul launch measured for itself: cycles of %clock64 over nanoseconds of %globaltimer,
+    both read by the first CTA at its start and end and left in the workspace header."""
+    import torch
+    cyc, ns = (int(v) for v in ws[48:64].view(torch.int64).tolist())
+    return 1e3 * cyc / ns if ns > 0 else None
+
 
 def run_ours(args):
     import torch
@@ -281,6 +391,7 @@ def run_ours(args):
         raise SystemExit("bench.py: no CUDA device — the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    gpu_index = _physical_gpu_index(local_rank)
     replicas.init("nccl", dev)
     api.lib()
     peaks = _peaks()
@@ -359,7 +470,7 @@ def run_ours(args):
         step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(_physical_gpu_index(local_rank)) as clk:
+    with ClockSampler(gpu_index) as clk:
         e0.record()
         for _ in range(args.steps):
             step()
@@ -370,11 +481,12 @@ def run_ours(args):
     if status != 0:
         raise SystemExit(f"bench.py: device-side status {status} ({api.status_string(status)})")
     value = world * FLOP_PER_STEP * args.steps / (ms * 1e-3) / 1e12
+    headline_kernel_mhz = _kernel_clock_mhz(ws)          # what the last launch of the timed region ran at
 
     # ---- roofline of the dominant kernel (the tcgen05 matmul), timed alone on the same operands ------
     # The three matmuls of a step are launched here on the already fake-quantized operands (format NONE
     # skips the quantizers), each launch bracketed by CUDA events on the launching stream.
-    achieved, gemm_ms = None, None
+    achieved, gemm_ms, gemm_mhz = None, None, None
     Xh = api.qf_qdq(fmt, X, want_codes=False, want_scales=False)["out"]
     Wh = api.qf_qdq(fmt, W, want_codes=False, want_scales=False)["out"]
     n_rep = max(3, min(args.steps, 20)) if "roofline" in sections else -2
@@ -395,7 +507,29 @@ def run_ours(args):
     if evs:
         gemm_ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
         achieved = FLOP_PER_GEMM / (gemm_ms * 1e-3) / 1e12
+        gemm_mhz = _kernel_clock_mhz(ws)
     del Xh, Wh
+
+    # ---- sustained: the same step back to back for at least two seconds (the power cap pulls the clock down) ----
+    sustained = None
+    if "sustained" in sections:
+        n_sus = max(args.steps, int(2000.0 / (ms / args.steps)) + 1)
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(gpu_index) as sclk:
+            s0.record()
+            for _ in range(n_sus):
+                step()
+            s1.record()
+            barrier()
+        sms = replicas.max_over_ranks(s0.elapsed_time(s1), dev)
+        sval = world * FLOP_PER_STEP * n_sus / (sms * 1e-3) / 1e12
+        smhz = _kernel_clock_mhz(ws)
+        sustained = {"value": sval, "unit": "TFLOP/s", "steps": n_sus, "seconds": sms * 1e-3, "ms_per_step": sms / n_sus,
+                     "clocks": sclk.summary(), "sm_mhz_in_kernel": smhz,
+                     "frac_of_measured_sustained": sval / world / peaks["bf16_sustained"],
+                     "frac_of_2250_datasheet": sval / world / DATASHEET_TFLOPS,
+                     "frac_of_tensor_peak_at_kernel_clock": (sval / world) / (NUM_SMS * TENSOR_FLOP_PER_CLK_PER_SM * smhz * 1e6 / 1e12) if smhz else None}
 
     # ---- end to end: host buffers, H2D of the inputs and D2H of the results inside the timed region ---
     # Every step copies X, W, dY from pinned host memory, runs the step through the C ABI, and copies
@@ -469,11 +603,13 @@ def run_ours(args):
     if rank == 0 and world == 1 and "configs" in sections:
         del X, W, dY, Y, dX, dW, ws
         torch.cuda.empty_cache()
-        other = measure_other_workloads(torch, api, synth, dev, peaks)
+        other = measure_other_workloads(torch, api, synth, dev, peaks, gpu_index)
 
     if rank == 0:
         clocks = clk.summary()
+        clocks["sm_mhz_in_kernel"] = headline_kernel_mhz
         peak = peaks["bf16_burst"]
+        at_clock = NUM_SMS * TENSOR_FLOP_PER_CLK_PER_SM * gemm_mhz * 1e6 / 1e12 if gemm_mhz else None
         line = {
             "metric": "fake-quant linear fwd+bwd TFLOPS", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -488,12 +624,18 @@ def run_ours(args):
             "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel (tcgen05 cta_group::2 BF16, 256x256x64 tiles per CTA pair)", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
                          # mean dram__bytes_read.sum + dram__bytes_write.sum per launch over the three matmuls of a
-                         # step, from an ncu capture of this workload (summary committed with the other profiles)
-                         "traffic": 916.2e6 if (M, N, K) == (8192, 12288, 4096) else None,
+                         # step, read from the committed ncu summary of this shape (None for other shapes)
+                         "traffic": _profiled_traffic(M, N, K),
+                         "algorithmic_bytes": (2.0 * (M * K + N * K) + 2.0 * M * N + 2.0 * (M * N + N * K) + 2.0 * M * K
+                                               + 2.0 * (M * N + M * K) + 4.0 * N * K) / 3.0,
                          "peak_source": f"{peaks['source']} cuBLAS bf16 burst", "ms_per_launch": gemm_ms,
+                         "sm_mhz_in_kernel": gemm_mhz,
+                         "frac_of_tensor_peak_at_kernel_clock": achieved / at_clock if achieved and at_clock else None,
                          "frac_of_sustained": achieved / peaks["bf16_sustained"] if achieved else None,
-                         "frac_of_2250_datasheet": achieved / 2250.0 if achieved else None,
-                         "step_frac_of_burst": value / world / peak},
+                         "frac_of_2250_datasheet": achieved / DATASHEET_TFLOPS if achieved else None,
+                         "step_frac_of_burst": value / world / peak,
+                         "step_frac_of_2250_datasheet": value / world / DATASHEET_TFLOPS},
+            "sustained": sustained,
             "cpu_baseline": cpu,
             "qdq_gbs": qdq,
         }
@@ -510,15 +652,22 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sections", default=",".join(SECTIONS),
-                    help="extra measurements beside the headline: roofline,qdq,e2e,cpu (default), configs = the other "
-                         "named workloads (empty string: none)")
+                    help="measurements beside the headline: roofline, sustained, qdq, e2e, cpu, configs (the other named "
+                         "workloads); all by default (empty string: none)")
     ap.add_argument("--shape", default=None, help="M,N,K of a smaller case (profiler captures only)")
     ap.add_argument("--in-kernel-qdq", action="store_true",
                     help="run the step with QF_FUSED_QDQ (quantize the staged tiles inside the matmul kernel) instead of the default path")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="launch and timing protocol only (gloo ranks that sleep; no GPU): checks that --gpus N starts N ranks")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under torchrun: start the ranks ourselves, one per GPU
+        raise SystemExit(spawn_ranks(args.gpus, sys.argv[1:]))
     if args.shape:
         _set_shape(args.shape)
-    if args.impl == "reference":
+    if args.dry_run:
+        run_dry(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

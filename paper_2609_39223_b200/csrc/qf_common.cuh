@@ -24,6 +24,8 @@ enum WsWord : int {
   kWsScaleW = 8,      // derived NVFP4 tensor scale of W (float)
   kWsScaleA = 9,      // derived NVFP4 tensor scale of X (float)
   kWsGuessW = 10,     // the caller's guess of W's tensor scale (float bits), kept for the conditional second pass
+  kWsClkCycles = 12,  // 64-bit: SM clock cycles the last matmul launch ran for (first CTA, start to end)
+  kWsClkNanos = 14,   // 64-bit: the same interval in nanoseconds of the global timer; cycles / ns = SM clock in GHz
 };
 
 // ---- device helpers -----------------------------------------------------------------------

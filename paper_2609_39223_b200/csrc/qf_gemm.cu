@@ -1,8 +1,11 @@
 // BF16 x BF16 -> FP32 matmul on the 5th-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory), operands staged by TMA into 128-byte-swizzled shared memory. One persistent CTA
-// per SM walks output tiles of 128 x 256; a 4-stage TMA ring feeds a single MMA-issuing thread;
-// the 512 TMEM columns hold two accumulators so the epilogue of one tile overlaps the main loop of
-// the next.
+// tensor memory), operands staged by TMA into 128-byte-swizzled shared memory. Two persistent kernels share
+// one pipeline design (a TMA ring feeding a single MMA-issuing thread; the 512 TMEM columns hold two
+// accumulators, so the epilogue of one tile overlaps the main loop of the next):
+//   gemm_pair_kernel  the main one: a cluster of two CTAs per 256 x 256 output tile, cta_group::2 MMAs, 6 stages,
+//                     optional in-kernel MXFP4 quantization of the staged tiles;
+//   gemm_kernel       one CTA per 128 x 256 tile, 4 stages: outputs with fewer than 256 rows, and grouped layers
+//                     with more experts than the pair kernel's shared-memory tile table holds.
 //
 // The three products of the quantization-aware layer (Eq. fakequant, Eq. ste, Eq. activation-ste)
 // differ only in which operand dimension is contiguous in memory:
@@ -54,7 +57,9 @@ struct KParams {
   int64_t Mo, No, Kc, ldc;
   int c_dtype, accumulate;
   int tiles_m, tiles_n, num_tiles;
-  int band;                  // row-tiles per rasterization band (see band_rows())
+  int band;                  // tiles per rasterization band along the banded dimension (see choose_raster())
+  int raster;                // 0: bands of row tiles, rows fastest inside a band (the band's A panels stay in L2, B streams);
+                             // 1: bands of column tiles, columns fastest (the band's B panels stay, A streams)
   int group_mode, G;
   const int32_t* offs;
   int64_t b_group_rows;      // mode 1: rows one group occupies in B's 2-D tensor map
@@ -296,6 +301,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  KernelClock kclock;
+  const bool clocked = blockIdx.x == 0 && threadIdx.x == 0;
+  if (clocked) kclock.start();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -446,6 +454,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
+  if (clocked) kclock.stop(p.status);
 }
 
 // =====================================================================================================
@@ -561,13 +570,24 @@ __device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum
     g = t / per;
     t -= g * per;
   }
-  const int band = p.band * p.tiles_n;
-  const int bidx = t / band;
-  const int first_m = bidx * p.band;
-  const int rows_in_band = min(p.band, tiles_m - first_m);
-  const int within = t - bidx * band;
-  const int mt = first_m + within % rows_in_band;
-  r.n0 = (within / rows_in_band) * BN;
+  int mt;
+  if (p.raster == 0) {
+    const int band = p.band * p.tiles_n;
+    const int bidx = t / band;
+    const int first_m = bidx * p.band;
+    const int rows_in_band = min(p.band, tiles_m - first_m);
+    const int within = t - bidx * band;
+    mt = first_m + within % rows_in_band;
+    r.n0 = (within / rows_in_band) * BN;
+  } else {
+    const int band = p.band * tiles_m;
+    const int bidx = t / band;
+    const int first_n = bidx * p.band;
+    const int cols_in_band = min(p.band, p.tiles_n - first_n);
+    const int within = t - bidx * band;
+    mt = within / cols_in_band;
+    r.n0 = (first_n + within % cols_in_band) * BN;
+  }
   r.m0 = mt * (2 * BM);
   if (p.group_mode == 1) {
     int lo = 0, hi = p.G;                     // invariant: cum[lo] <= mt < cum[hi]
@@ -644,8 +664,9 @@ __device__ __forceinline__ void mxfp4_transform_tile(uint32_t base, int warp_in_
 }
 
 // FUSE: bit 0 = quantize-dequantize the staged A tile (MXFP4), bit 1 = the staged B tile. With FUSE != 0
-// eight extra warps transform each stage in shared memory between the TMA arrival and the MMA issue, so
-// the fake-quantized operand never exists in global memory.
+// TRANSFORM_WARPS extra warps (sixteen, in four groups that take alternate k-blocks) transform each stage in
+// shared memory between the TMA arrival and the MMA issue, so the fake-quantized operand never exists in
+// global memory.
 template <bool A_MN, bool B_MN, typename OutT, int FUSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FUSE ? NUM_THREADS_FUSED : NUM_THREADS, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -664,6 +685,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const bool leader = rank == 0;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
+  KernelClock kclock;
+  const bool clocked = blockIdx.x == 0 && threadIdx.x == 0;
+  if (clocked) kclock.start();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) {
@@ -869,6 +893,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
+  if (clocked) kclock.stop(p.status);
 }
 
 // Self-test of the bounded wait: one thread waits on a barrier that nothing will ever arrive at, with a
@@ -911,6 +936,25 @@ int band_rows(int64_t tile_rows, int64_t Kc, int tiles_m) {
   if (band > 32) band = 32;
   if (band > tiles_m) band = tiles_m;
   return static_cast<int>(band < 1 ? 1 : band);
+}
+
+// Rasterization of plain problems on the two-CTA kernel. Tiles are walked in bands along one output dimension, the
+// banded dimension fastest: the band's operand panels are re-read by every wave and stay in L2, the other operand
+// streams past once per band. DRAM traffic is then about  banded + other * (number of bands),  so the SMALLER operand is
+// the one to band (the product term is the same either way, the additive term is the banded operand). A band of panels
+// is kept near 50 MB (measured on B200 with ncu at 8192 x 12288 x 4096: beyond that the band no longer survives in
+// the 126 MB L2 and traffic doubles; hints to evict the streaming operand first made things worse, since that operand
+// is shared by the CTAs of a wave), and the bands are made equal. Measured DRAM bytes per launch with this choice against
+// row bands of 40 MB for every product: forward 514 vs 526 MB, dgrad 912 vs 1131 MB, wgrad 978 vs 1158 MB.
+void choose_raster(int64_t Mo, int64_t No, int64_t Kc, int tiles_m, int tiles_n, int* raster, int* band) {
+  const bool band_cols = No < Mo;                                   // B (No x Kc) is the smaller operand
+  const int tiles = band_cols ? tiles_n : tiles_m;
+  const int64_t panel = 256 * (Kc > 0 ? Kc : 1) * 2;                // bytes of one 256-wide operand panel
+  int64_t band_max = (52ll << 20) / panel;
+  if (band_max < 4) band_max = 4;
+  const int64_t nbands = (tiles + band_max - 1) / band_max;
+  *raster = band_cols ? 1 : 0;
+  *band = static_cast<int>((tiles + nbands - 1) / nbands);
 }
 
 // 3-D tensor map over the output for the epilogue's TMA stores: [groups, rows, cols] with a
@@ -1026,6 +1070,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.num_tiles = kp.tiles_m * kp.tiles_n * (a.group_mode == 2 ? a.G : 1);
   const int64_t contraction_rows = a.group_mode == 2 ? a.rows_padded : a.Kc;
   kp.band = band_rows(2 * BM, a.group_mode == 2 ? a.rows_padded / (a.G > 0 ? a.G : 1) : a.Kc, kp.tiles_m);
+  if (a.group_mode == 0) choose_raster(a.Mo, a.No, a.Kc, kp.tiles_m, kp.tiles_n, &kp.raster, &kp.band);
   CUtensorMap tmA, tmB;
   bool ok;
   if (a.a_mn_major) ok = make_map(&tmA, a.A, contraction_rows, a.Mo, a.lda, 64, BK);

@@ -48,6 +48,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// Read-only counters for reporting the clock a kernel actually ran at (nothing is set or changed).
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+struct KernelClock {
+  long long c0;
+  unsigned long long t0;
+  __device__ __forceinline__ void start() { c0 = clock64(); t0 = globaltimer_ns(); }
+  // status points at the first word of the workspace header
+  __device__ __forceinline__ void stop(uint32_t* status) const {
+    if (!status) return;
+    unsigned long long* w = reinterpret_cast<unsigned long long*>(status + kWsClkCycles);
+    w[0] = static_cast<unsigned long long>(clock64() - c0);
+    w[1] = globaltimer_ns() - t0;
+  }
+};
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

@@ -2,9 +2,10 @@
 // formats; Eq. nvfp4 / mxfp4 / q4k and their dequantization equations), plus the tensor-amax
 // pre-pass NVFP4 needs and the stand-alone dequantizers.
 //
-// Work decomposition: one thread owns one 16-byte chunk (8 BF16 values); a warp reads 512
-// contiguous bytes per load instruction. A quantization block is 2 (NVFP4), 4 (MXFP4) or 32
-// (Q4_K super-block) neighbouring lanes, so block statistics are warp shuffles. Every FP32
+// Work decomposition: FP4 formats: a lane owns 16 consecutive elements (two 16-byte loads): a whole
+// NVFP4 block, or half an MXFP4 block (one shuffle with the neighbouring lane). Q4_K: a lane owns one
+// 32-weight sub-block (four 16-byte loads), eight neighbouring lanes a super-block, whose statistics are
+// warp shuffles. The tensor-amax pass reads one 16-byte chunk per lane and load. Every FP32
 // operation that decides a code is written with an explicit round-to-nearest intrinsic so that
 // the compiler can neither contract it into an FMA nor replace a division by a reciprocal.
 #include "qf_common.cuh"
@@ -768,12 +769,14 @@ cudaError_t launch_amax(const void* in, int64_t n, uint32_t* amax_bits, cudaStre
 // ---- batched launches --------------------------------------------------------------------------------
 // Many tensors per call (every linear weight of a model is quantized each step for weight synchronisation, Section 3.4):
 // MXFP4, Q4_K and NVFP4 with supplied scales take one launch per 64 tensors. NVFP4 with derived scales needs every
-// tensor's maximum before its blocks can be scaled; the batch is cut into sub-batches small enough to stay in L2
-// (kSubBatchBytes of input), and launch j quantizes sub-batch j-1 while its spare y-slices take the maxima of
-// sub-batch j: S + 1 launches for S sub-batches instead of three per tensor, with the second read of every tensor
-// served from L2. With speculated scales (the previous step's) one launch quantizes with the guesses and gathers the
+// tensor's maximum before its blocks can be scaled; the batch is cut into sub-batches of kSubBatchBytes of input, and
+// launch j quantizes sub-batch j-1 while its spare y-slices take the maxima of sub-batch j: S + 1 launches for S
+// sub-batches instead of three per tensor, with part of the second read of every tensor served from L2. With speculated scales (the previous step's) one launch quantizes with the guesses and gathers the
 // true maxima, a second one derives the scales and requantizes only the tensors whose guess was wrong.
-constexpr int64_t kSubBatchBytes = 24ll << 20;
+// Measured on B200 with 32 tensors of 8 MB: the rate climbs with the sub-batch size up to about 40 MB (fewer launches) and is
+// flat from there to 128 MB (3.9-4.2 TB/s); six resident blocks per SM beat four and sixteen.
+constexpr int64_t kSubBatchBytes = 56ll << 20;
+constexpr int kBatchBlocksPerSm = 6;
 
 static int batched_grid_x(int64_t max_items, int per_thread, int ny, int blocks_per_sm) {
   int64_t gx = (max_items + static_cast<int64_t>(kThreads) * per_thread - 1) / (static_cast<int64_t>(kThreads) * per_thread);
@@ -851,7 +854,7 @@ cudaError_t launch_qdq_batched(const QdqBatchArgs& a, cudaStream_t st) {
       if (am.nchunks[i] > ma) ma = am.nchunks[i];
     }
     const int ny = prev_cnt + cnt;
-    const int64_t gq = batched_grid_x(mq, kUnitsPerThread, ny, 16), ga = batched_grid_x(ma, 4, ny, 16);
+    const int64_t gq = batched_grid_x(mq, kUnitsPerThread, ny, kBatchBlocksPerSm), ga = batched_grid_x(ma, 4, ny, kBatchBlocksPerSm);
     qdq_fp4_batched_kernel<QF_FMT_NVFP4><<<dim3(static_cast<unsigned>(gq > ga ? gq : ga), ny), kThreads, 0, st>>>(
         q, prev_cnt, am, nullptr, a.ws_words + prev0, a.tscales + prev0, 0, nullptr, nullptr, nullptr, a.ws_words + t);
     if (cudaError_t e = cudaGetLastError()) return e;
