@@ -71,10 +71,15 @@ typedef enum {
                                       recomputation. The paper's layer discards these copies after the forward matmul and
                                       recomputes them; keeping the workspace alive trades that memory for two passes. */
 #define QF_AMAX_RUNNING 0x10u      /* qf_nvfp4_tensor_scale: the incoming *amax_state takes part in the maximum        */
-#define QF_FUSED_QDQ 0x8u          /* linear calls: quantize-dequantize MXFP4 operands inside the matmul kernel, on the
-                                      tiles staged in shared memory, instead of writing fake-quantized copies to the
-                                      workspace first. Same results bit for bit. Applies to MXFP4 operands of
-                                      non-grouped calls with M >= 256; anything else silently takes the default path. */
+#define QF_FUSED_QDQ 0x8u          /* linear calls: quantize-dequantize MXFP4 and NVFP4 operands inside the matmul kernel,
+                                      on the tiles staged in shared memory, instead of writing fake-quantized copies to
+                                      the workspace first (Eq. fakequant: W_hat and A_hat are transient). Same results
+                                      bit for bit. An NVFP4 operand's tensor scale is settled before the launch (supplied,
+                                      or derived by a maximum pass over the operand; a speculated scale is derived).
+                                      Applies to plain and grouped calls with at least 256 output rows (and at most 256
+                                      experts); Q4_K weights (a super-block spans four staged tiles) and anything else
+                                      silently take the default path. Slower than the default on B200 at every shape
+                                      measured: an option, not the default. */
 
 #define QF_MXFP4_NO_CLIP 0x80u      /* qf_qdq, qf_qdq_lora and the linear calls: MXFP4 block exponent p = the smallest one
                                       with amax <= 6 * 2^p (nothing saturates) instead of floor(log2 amax) - 2, under

@@ -88,6 +88,25 @@ qf_status_t quantize_operand(int fmt, const void* src, int64_t rows, int64_t col
   return cu(launch_qdq(q, st));
 }
 
+// Tensor scale(s) of an NVFP4 operand that the matmul kernel quantizes itself (QF_FUSED_QDQ): *out receives a device
+// pointer to the final scale(s) - the caller's when given, otherwise derived now from the operand's maximum (and written
+// back to the caller's array when there is one), with the maximum left in header[amax_word] for single tensors.
+qf_status_t fused_nvfp4_scale(const void* src, int64_t rows, int64_t cols, float* tscale_user, bool given, uint32_t* header,
+                              int amax_word, int scale_word, int groups, cudaStream_t st, const float** out) {
+  if (given) { *out = tscale_user; return QF_OK; }
+  QdqArgs q{};
+  q.fmt = QF_FMT_NVFP4;
+  q.in = src;
+  q.rows = rows;
+  q.cols = cols;
+  q.groups = groups;
+  q.tscale_out = tscale_user ? tscale_user : reinterpret_cast<float*>(header + scale_word);
+  *out = q.tscale_out;
+  return cu(launch_nvfp4_scales_only(q, header, amax_word, st));
+}
+
+inline bool fusable_fmt(int fmt) { return fmt == QF_FMT_MXFP4 || fmt == QF_FMT_NVFP4; }
+
 // Checks shared by the forward and backward calls. W may be NULL only when the caller does not need it
 // (a backward call that asks for dW alone): need_w says whether it is required.
 qf_status_t check_linear_common(const void* W, bool need_w, int64_t M, int64_t N, int64_t K, int wq, int aq, const float* w_ts,
@@ -139,33 +158,39 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
     g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M;
   }
   const bool may_fuse = (flags & QF_FUSED_QDQ) && gemm_can_fuse(g);
-  g.fuse_b_mxfp4 = may_fuse && wq == QF_FMT_MXFP4;
-  g.fuse_a_mxfp4 = may_fuse && aq == QF_FMT_MXFP4;
+  const bool fuse_b = may_fuse && fusable_fmt(wq) && !(flags & QF_REUSE_W_HAT);
+  const bool fuse_a = may_fuse && fusable_fmt(aq) && !(flags & QF_REUSE_X_HAT);
   const void* Wh = W;
   const void* Xh = X;
-  if (K > 0) {
-    if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
-      if (!(flags & QF_REUSE_W_HAT))
-        if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
-      Wh = w.w_hat;
-    }
-    // max|X| for the caller's running maximum: taken from the quantize pass over X where there is one (its own
-    // accumulator for a single-pass FP4 quantizer, the derive path's maximum word for NVFP4 without a supplied
-    // scale), otherwise from a pass of its own
-    const bool x_pass = aq != QF_FMT_NONE && !g.fuse_a_mxfp4 && !(flags & QF_REUSE_X_HAT);
-    const bool x_derives = x_pass && aq == QF_FMT_NVFP4 && !(flags & QF_A_TSCALE_GIVEN);
-    const bool x_accumulates = x_pass && !x_derives && (aq == QF_FMT_NVFP4 || aq == QF_FMT_MXFP4);
-    uint32_t* amax_word = a_amax_out ? (x_derives ? w.header + kWsAmaxA : w.header + kWsAmaxReport) : nullptr;
-    if (a_amax_out && !x_derives && !x_accumulates)
-      if (cudaError_t e = launch_amax(X, M * K, amax_word, st)) return cu(e);
-    if (aq != QF_FMT_NONE && !g.fuse_a_mxfp4) {
-      if (!(flags & QF_REUSE_X_HAT))
-        if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0, false, (a_amax_out && x_accumulates) ? amax_word : nullptr)) return s;
-      Xh = w.x_hat;
-    }
-    if (a_amax_out)
-      if (cudaError_t e = launch_amax_to_float(amax_word, a_amax_out, st)) return cu(e);
+  if (fuse_b) {
+    g.fuse_b_fmt = wq;
+    g.fuse_b_tscale_per_group = groups > 1;
+    if (wq == QF_FMT_NVFP4)
+      if (qf_status_t s = fused_nvfp4_scale(W, groups * N, K, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, static_cast<int>(groups), st, &g.fuse_b_tscale)) return s;
+  } else if (wq != QF_FMT_NONE) {
+    if (!(flags & QF_REUSE_W_HAT))
+      if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
+    Wh = w.w_hat;
   }
+  // max|X| for the caller's running maximum: taken from the pass that derives X's NVFP4 scale (its maximum word) or from
+  // the single-pass FP4 quantizer over X (its own accumulator) where there is one, otherwise from a pass of its own
+  const bool x_pass = aq != QF_FMT_NONE && !fuse_a && !(flags & QF_REUSE_X_HAT);
+  const bool x_derives = aq == QF_FMT_NVFP4 && !(flags & QF_A_TSCALE_GIVEN) && (x_pass || fuse_a);
+  const bool x_accumulates = x_pass && !x_derives && (aq == QF_FMT_NVFP4 || aq == QF_FMT_MXFP4);
+  uint32_t* amax_word = a_amax_out ? (x_derives ? w.header + kWsAmaxA : w.header + kWsAmaxReport) : nullptr;
+  if (a_amax_out && !x_derives && !x_accumulates)
+    if (cudaError_t e = launch_amax(X, M * K, amax_word, st)) return cu(e);
+  if (fuse_a) {
+    g.fuse_a_fmt = aq;
+    if (aq == QF_FMT_NVFP4)
+      if (qf_status_t s = fused_nvfp4_scale(X, M, K, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, 1, st, &g.fuse_a_tscale)) return s;
+  } else if (aq != QF_FMT_NONE) {
+    if (!(flags & QF_REUSE_X_HAT))
+      if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0, false, (a_amax_out && x_accumulates) ? amax_word : nullptr)) return s;
+    Xh = w.x_hat;
+  }
+  if (a_amax_out)
+    if (cudaError_t e = launch_amax_to_float(amax_word, a_amax_out, st)) return cu(e);
   g.A = Xh; g.B = Wh;
   return cu(launch_gemm(g, st));
 }
@@ -203,9 +228,14 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.status_word = w.header + kWsStatus;
   g.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
     if (grouped) { g.group_mode = 1; g.group_offsets = offs; g.G = G; g.rows_padded = M; }
-    g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && wq == QF_FMT_MXFP4 && gemm_can_fuse(g);
+    const bool fuse_b = (flags & QF_FUSED_QDQ) && fusable_fmt(wq) && !(flags & QF_REUSE_W_HAT) && gemm_can_fuse(g);
     const void* Wh = W;
-    if (wq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
+    if (fuse_b) {
+      g.fuse_b_fmt = wq;
+      g.fuse_b_tscale_per_group = groups > 1;
+      if (wq == QF_FMT_NVFP4)
+        if (qf_status_t s = fused_nvfp4_scale(W, groups * N, K, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, static_cast<int>(groups), st, &g.fuse_b_tscale)) return s;
+    } else if (wq != QF_FMT_NONE) {
       if (!(flags & QF_REUSE_W_HAT))
         if (qf_status_t s = quantize_operand(wq, W, groups * N, K, w.w_hat, w_ts, flags & QF_W_TSCALE_GIVEN, w.header, kWsAmaxW, kWsScaleW, st, static_cast<int>(groups), (flags & QF_MXFP4_NO_CLIP) != 0, (flags & QF_W_TSCALE_SPECULATIVE) != 0)) return s;
       Wh = w.w_hat;
@@ -225,9 +255,13 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     g.status_word = w.header + kWsStatus;
   g.mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
     if (grouped) { g.group_mode = 2; g.group_offsets = offs; g.G = G; g.rows_padded = M; g.c_group_stride = N * K; }
-    g.fuse_b_mxfp4 = (flags & QF_FUSED_QDQ) && aq == QF_FMT_MXFP4 && gemm_can_fuse(g);
+    const bool fuse_b = (flags & QF_FUSED_QDQ) && fusable_fmt(aq) && !(flags & QF_REUSE_X_HAT) && gemm_can_fuse(g);
     const void* Xh = X;
-    if (aq != QF_FMT_NONE && !g.fuse_b_mxfp4) {
+    if (fuse_b) {
+      g.fuse_b_fmt = aq;                 // the activations are this product's B operand; one scale for all of X
+      if (aq == QF_FMT_NVFP4)
+        if (qf_status_t s = fused_nvfp4_scale(X, M, K, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, 1, st, &g.fuse_b_tscale)) return s;
+    } else if (aq != QF_FMT_NONE) {
       if (!(flags & QF_REUSE_X_HAT))
         if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Xh = w.x_hat;

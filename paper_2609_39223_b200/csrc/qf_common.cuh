@@ -119,6 +119,106 @@ __device__ __forceinline__ uint32_t mxfp4_qdq_pair_bf16(uint32_t w, uint32_t one
   return bf2_bits(r) | (w & 0x80008000u);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Exact division without the per-element IEEE divide sequence.
+//
+// The formats need v = x / S (NVFP4) and t = (x + em) / es (Q4_K) as correctly rounded FP32
+// quotients, because the quotient decides a code. One divisor serves a whole block, so its correctly
+// rounded reciprocal rc = RN(1/y) is computed once and every quotient is then
+//     q0 = RN(x * rc);  q1 = RN(q0 + rc * (x - y*q0))          (x - y*q0 is exact in a fused multiply-add)
+// (two elements per instruction). With an exactly rounded reciprocal and no overflow / underflow in
+// the residual, q1 is the correctly rounded quotient (Markstein's division theorem); the range guard
+// below keeps operands where that holds and the caller falls back to the IEEE divide otherwise.
+// qf_selftest_div compares it with the IEEE divide (tens of billions of pairs, including every BF16
+// numerator and divisors with an all-ones significand, without a difference).
+//
+// The residual is formed rounding toward minus infinity. Being exact, its value does not depend on the
+// rounding mode, but its sign when it is zero does: an exactly cancelling sum is -0 in that mode, so the
+// correction step adds -0 to q0 and leaves q0's sign alone. That makes x = -0 come out as -0, like the
+// IEEE quotient (with round-to-nearest the residual would be +0 and (+0) + (-0) = +0).
+// ---------------------------------------------------------------------------------------------
+
+#ifndef QF_DIV_STEPS
+#define QF_DIV_STEPS 1      // residual corrections after the first product (1 suffices with an exact reciprocal)
+#endif
+
+
+__device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
+  const float2 ny = splat(-y), r = splat(rc);
+  float2 q = __fmul2_rn(x, r);
+  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
+#if QF_DIV_STEPS > 1
+  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
+#endif
+  return q;
+}
+__device__ __forceinline__ float div1_fast(float x, float y, float rc) {
+  float q = __fmul_rn(x, rc);
+  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
+#if QF_DIV_STEPS > 1
+  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
+#endif
+  return q;
+}
+// divisor magnitudes for which the iteration above is used
+__device__ __forceinline__ bool div_safe(float y) { return y >= 0x1p-60f && y <= 0x1p60f; }
+
+// NVFP4 per-tensor constants derived from the tensor scale: the divisor 6 * s_t of the block-scale quotient and its
+// exactly rounded reciprocal (when the divisor lies in the range where the reciprocal-based division is exact).
+struct Nvfp4Tensor {
+  float s_t, denom, rc_denom;
+  bool denom_safe;
+};
+__device__ __forceinline__ Nvfp4Tensor nvfp4_tensor(float s_t) {
+  Nvfp4Tensor t;
+  t.s_t = s_t;
+  t.denom = __fmul_rn(6.0f, s_t);
+  t.denom_safe = div_safe(t.denom);
+  t.rc_denom = t.denom_safe ? __frcp_rn(t.denom) : 0.0f;
+  return t;
+}
+
+// NVFP4 quantize-dequantize of NW packed BF16 pairs that belong to one 16-element block whose max |x| is amax_b
+// (Eq. nvfp4, Eq. nvfp4-dequant): block scale sb = E4M3(min(amax_b / (6 s_t), 448)), S = s_t * sb, codes from
+// x / S (the correctly rounded quotient by either route), x_hat = bf16((sb * value(code)) * s_t). `scale_code`
+// receives the E4M3 code and `codes` one byte per pair (low nibble = first element). Both division routes give the
+// IEEE quotient, so the choice between them never changes a result.
+template <int NW>
+__device__ __forceinline__ void nvfp4_block_words(const uint32_t (&w)[NW], float amax_b, const Nvfp4Tensor nt, uint32_t (&xhat)[NW],
+                                                  uint32_t (&codes)[NW], uint32_t& scale_code) {
+  // A supplied tensor scale can be far too small for a block: the quotient then exceeds every E4M3 value and may
+  // even overflow FP32, which the reciprocal-based form does not survive (inf - inf). 512 * denom is exact there;
+  // at or beyond it the scale is the largest code whatever the quotient.
+  const bool fast = nt.denom_safe && (amax_b == 0.0f || amax_b >= 0x1p-60f);
+  const float q = fast ? (amax_b >= __fmul_rn(512.0f, nt.denom) ? 512.0f : div1_fast(amax_b, nt.denom, nt.rc_denom))
+                       : __fdiv_rn(amax_b, nt.denom);
+  scale_code = e4m3_encode(q);
+  const float sb = e4m3_decode(scale_code);
+  const float S = __fmul_rn(nt.s_t, sb);
+  const float2 sb2 = splat(sb), st2 = splat(nt.s_t);
+  if (S == 0.0f) {
+#pragma unroll
+    for (int j = 0; j < NW; ++j) { xhat[j] = 0u; codes[j] = 0u; }
+  } else if (fast && div_safe(S) && amax_b <= __fmul_rn(8.0f, S)) {
+    const float rc = __frcp_rn(S);
+#pragma unroll
+    for (int j = 0; j < NW; ++j) {
+      const float2 v = div2_fast(unpack2(w[j]), S, rc);
+      codes[j] = e2m1x2_encode(v.x, v.y);
+      const float2 o = __fmul2_rn(__fmul2_rn(sb2, e2m1x2_decode(codes[j])), st2);
+      xhat[j] = pack_bf16x2(o.x, o.y);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < NW; ++j) {
+      const float2 x = unpack2(w[j]);
+      codes[j] = e2m1x2_encode(__fdiv_rn(x.x, S), __fdiv_rn(x.y, S));
+      const float2 o = __fmul2_rn(__fmul2_rn(sb2, e2m1x2_decode(codes[j])), st2);
+      xhat[j] = pack_bf16x2(o.x, o.y);
+    }
+  }
+}
+
 // ---- host-side launchers implemented in the .cu files ---------------------------------------
 
 // NVFP4 with a speculated tensor scale: the first pass quantizes with the caller's guess while it accumulates the true
@@ -173,6 +273,8 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
 cudaError_t launch_amax_to_scale(const uint32_t* amax_bits, float* scale, cudaStream_t st);
 cudaError_t launch_qdq(const QdqArgs& a, cudaStream_t st);
 cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st);
+// the first half of that alone: *a.tscale_out (a.groups floats) receives the derived tensor scale(s); nothing is quantized
+cudaError_t launch_nvfp4_scales_only(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st);
 cudaError_t launch_dequant(int fmt, const void* codes, const void* scales, const float* tscale, int64_t rows,
                            int64_t cols, void* out, cudaStream_t st);
 cudaError_t launch_selftest_div(const float* xs, int64_t nx, const float* ys, int64_t ny, unsigned long long* mismatches,
@@ -201,8 +303,12 @@ struct GemmArgs {
   int64_t c_group_stride;        // elements between consecutive groups of C (mode 2)
   int64_t rows_padded;           // mode 1: total rows of A / C; mode 2: total contraction rows
   uint32_t* status_word;         // device word receiving QF_ERR_TIMEOUT if a wait expires
-  bool fuse_a_mxfp4, fuse_b_mxfp4;   // apply the MXFP4 quantize-dequantize to the staged tiles inside the kernel
-  bool mxfp4_noclip;                 // scale rule of that in-kernel quantizer (QF_MXFP4_NO_CLIP)
+  int fuse_a_fmt, fuse_b_fmt;        // QF_FMT_MXFP4 / QF_FMT_NVFP4: quantize-dequantize the staged tiles of that operand
+                                     // inside the kernel (QF_FMT_NONE: the operand is used as it is)
+  const float* fuse_a_tscale;        // NVFP4: device tensor scale of A (one float), final before the launch
+  const float* fuse_b_tscale;        // NVFP4: device tensor scale(s) of B: one float, or one per group (mode 1)
+  bool fuse_b_tscale_per_group;
+  bool mxfp4_noclip;                 // scale rule of the in-kernel MXFP4 quantizer (QF_MXFP4_NO_CLIP)
 };
 
 cudaError_t launch_pack_q4k(const void* codes, const void* scales, int64_t nsb, void* records, bool unpack, void* codes_out,

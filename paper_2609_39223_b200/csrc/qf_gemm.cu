@@ -66,6 +66,10 @@ struct KParams {
   int64_t c_group_stride;    // mode 2: elements between per-group outputs
   uint32_t* status;
   int mxfp4_noclip;          // scale rule of the in-kernel MXFP4 quantizer
+  int fuse_a_fmt, fuse_b_fmt;        // format of the in-kernel quantizer per operand (QF_FMT_MXFP4 / QF_FMT_NVFP4)
+  const float* a_tscale;             // NVFP4 in-kernel quantizer: tensor scale of A
+  const float* b_tscale;             // ... of B: one value, or one per group (grouped mode 1)
+  int b_tscale_per_group;
 };
 
 // ---- descriptors ------------------------------------------------------------------------------
@@ -551,6 +555,7 @@ struct PairTile {
   int b_row_off;         // mode 1: row offset of this tile's expert in B's 2-D tensor map
   int z;                 // mode 2: which per-expert output matrix
   int rows_limit;        // output rows at or beyond this index do not belong to this tile's matrix / segment
+  int group;             // mode 1: the expert whose weights this tile multiplies by (0 otherwise)
 };
 
 // Pair tiles are walked row-tile fastest inside bands (see band_rows()). Grouped mode 1: the row-tile
@@ -563,6 +568,7 @@ __device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum
   r.k_end = static_cast<int>(p.Kc);
   r.b_row_off = 0;
   r.z = 0;
+  r.group = 0;
   r.rows_limit = static_cast<int>(p.Mo);
   int g = 0;
   if (p.group_mode == 2) {
@@ -598,6 +604,7 @@ __device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum
     r.m0 = group_off(p, lo) + (mt - cum[lo]) * (2 * BM);
     r.rows_limit = group_off(p, lo + 1);
     r.b_row_off = lo * static_cast<int>(p.b_group_rows);
+    r.group = lo;
   } else if (p.group_mode == 2) {
     r.k_begin = group_off(p, g);
     r.k_end = group_off(p, g + 1);
@@ -663,7 +670,40 @@ __device__ __forceinline__ void mxfp4_transform_tile(uint32_t base, int warp_in_
   for (int b = 0; b < PER_WARP / (32 * BATCH); ++b) mxfp4_transform_batch<BATCH>(slab + static_cast<uint32_t>(b) * (32u * BATCH * 16u), noclip);
 }
 
-// FUSE: bit 0 = quantize-dequantize the staged A tile (MXFP4), bit 1 = the staged B tile. With FUSE != 0
+// The same for NVFP4 (Eq. nvfp4 with the tensor scale already final): a 16-element block is an aligned PAIR of 16-byte
+// chunks, which the swizzle also maps onto an aligned pair, so lanes l and l ^ 1 hold one block and combine their maxima
+// with one shuffle. Arithmetic identical to the stand-alone quantizer (nvfp4_block_words): same bits.
+template <int PER>
+__device__ __forceinline__ void nvfp4_transform_batch(uint32_t slab, const Nvfp4Tensor nt) {
+  uint4 v[PER];
+  uint32_t m[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) v[i] = ld_shared_v4(slab + static_cast<uint32_t>(i) * 512u);
+#pragma unroll
+  for (int i = 0; i < PER; ++i) m[i] = chunk8_amax_bits(v[i].x, v[i].y, v[i].z, v[i].w);
+#pragma unroll
+  for (int i = 0; i < PER; ++i) m[i] = max(m[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], 1));
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+    uint32_t o[4], codes[4], scale_code;
+    nvfp4_block_words<4>(w, __uint_as_float(m[i] << 16), nt, o, codes, scale_code);
+    st_shared_v4(slab + static_cast<uint32_t>(i) * 512u, o[0], o[1], o[2], o[3]);
+  }
+}
+
+template <int NCHUNKS>
+__device__ __forceinline__ void nvfp4_transform_tile(uint32_t base, int warp_in_group, int lane, const Nvfp4Tensor nt) {
+  constexpr int PER_WARP = NCHUNKS / WARPS_PER_GROUP;
+  constexpr int BATCH = 2;
+  static_assert(PER_WARP % (32 * BATCH) == 0, "tile must split evenly");
+  const uint32_t slab = base + static_cast<uint32_t>(warp_in_group * PER_WARP + lane) * 16u;
+#pragma unroll 1
+  for (int b = 0; b < PER_WARP / (32 * BATCH); ++b) nvfp4_transform_batch<BATCH>(slab + static_cast<uint32_t>(b) * (32u * BATCH * 16u), nt);
+}
+
+// FUSE: bit 0 = quantize-dequantize the staged A tile, bit 1 = the staged B tile (format per operand at run time:
+// MXFP4 or NVFP4). With FUSE != 0
 // TRANSFORM_WARPS extra warps (sixteen, in four groups that take alternate k-blocks) transform each stage in
 // shared memory between the TMA arrival and the MMA issue, so the fake-quantized operand never exists in
 // global memory.
@@ -814,8 +854,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int group = twarp / WARPS_PER_GROUP, wig = twarp % WARPS_PER_GROUP;
     uint32_t it = 0;                                  // running k-block count over all of this CTA's tiles
     bool alive = true;
+    const bool a_nv = (FUSE & 1) && p.fuse_a_fmt == QF_FMT_NVFP4, b_nv = (FUSE & 2) && p.fuse_b_fmt == QF_FMT_NVFP4;
+    const Nvfp4Tensor nt_a = nvfp4_tensor(a_nv ? __ldg(p.a_tscale) : 1.0f);
     for (int t = cluster_id; t < num_tiles && alive; t += num_clusters) {
       const PairTile tile = decode_pair(p, cum, tiles_m, t);
+      const Nvfp4Tensor nt_b = nvfp4_tensor(b_nv ? __ldg(p.b_tscale + (p.b_tscale_per_group ? tile.group : 0)) : 1.0f);
       for (int k = tile.k_begin; k < tile.k_end; k += BK, ++it) {
         if (static_cast<int>(it % TRANSFORM_GROUPS) != group) continue;
         const uint32_t stage = it % STAGES2, phase = (it / STAGES2) & 1u;
@@ -831,8 +874,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         got = __shfl_sync(0xFFFFFFFFu, got, 0);
         if (!got) { alive = false; break; }
         const uint32_t a_addr = tiles_base + stage * STAGE2_BYTES;
-        if (FUSE & 1) mxfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane, p.mxfp4_noclip != 0);
-        if (FUSE & 2) mxfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane, p.mxfp4_noclip != 0);
+        if (FUSE & 1) {
+          if (a_nv) nvfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane, nt_a);
+          else mxfp4_transform_tile<A2_BYTES / 16>(a_addr, wig, lane, p.mxfp4_noclip != 0);
+        }
+        if (FUSE & 2) {
+          if (b_nv) nvfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane, nt_b);
+          else mxfp4_transform_tile<B2_BYTES / 16>(a_addr + A2_BYTES, wig, lane, p.mxfp4_noclip != 0);
+        }
         fence_async_smem();                          // make the generic-proxy writes visible to the tensor core
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->ready[stage]), 0));
@@ -1009,7 +1058,7 @@ cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const 
 template <typename OutT>
 cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
                                const KParams& kp, int grid, cudaStream_t st) {
-  const int fuse = (a.fuse_a_mxfp4 ? 1 : 0) | (a.fuse_b_mxfp4 ? 2 : 0);
+  const int fuse = (a.fuse_a_fmt ? 1 : 0) | (a.fuse_b_fmt ? 2 : 0);
   if (!a.a_mn_major && !a.b_mn_major) {
     if (fuse == 3) return launch_pair_t<false, false, OutT, 3>(tmA, tmB, tmC, kp, grid, st);
     if (fuse == 2) return launch_pair_t<false, false, OutT, 2>(tmA, tmB, tmC, kp, grid, st);
@@ -1058,6 +1107,11 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.accumulate = a.accumulate ? 1 : 0;
   kp.status = a.status_word;
   kp.mxfp4_noclip = a.mxfp4_noclip ? 1 : 0;
+  kp.fuse_a_fmt = a.fuse_a_fmt;
+  kp.fuse_b_fmt = a.fuse_b_fmt;
+  kp.a_tscale = a.fuse_a_tscale;
+  kp.b_tscale = a.fuse_b_tscale;
+  kp.b_tscale_per_group = a.fuse_b_tscale_per_group ? 1 : 0;
   kp.group_mode = a.group_mode;
   kp.G = a.G;
   kp.offs = a.group_offsets;
@@ -1094,9 +1148,6 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   return launch_pair_majors<__nv_bfloat16>(a, tmA, tmB, tmC, kp, grid, st);
 }
 
-// True if launch_gemm would run this problem on the kernel that can quantize-dequantize staged tiles itself.
-bool gemm_can_fuse(const GemmArgs& a) { return a.group_mode == 0 && a.Mo >= 2 * BM && a.Kc > 0; }
-
 // Problems the two-CTA kernel takes: plain ones with at least one full 256-row tile, and grouped ones
 // whose expert count fits its shared-memory tile table (segments start on multiples of 128 rows).
 static bool pair_applies(const GemmArgs& a) {
@@ -1107,10 +1158,14 @@ static bool pair_applies(const GemmArgs& a) {
   return a.Mo >= 2 * BM && a.rows_padded > 0;
 }
 
+// True if launch_gemm would run this problem on the kernel that can quantize-dequantize staged tiles itself
+// (plain and grouped problems alike: the transform works on whatever tile the producer staged).
+bool gemm_can_fuse(const GemmArgs& a) { return pair_applies(a); }
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
   if (pair_applies(a)) return launch_gemm_pair(a, st);
-  if (a.fuse_a_mxfp4 || a.fuse_b_mxfp4) return cudaErrorInvalidValue;       // only the two-CTA kernel fuses (see gemm_can_fuse)
+  if (a.fuse_a_fmt || a.fuse_b_fmt) return cudaErrorInvalidValue;           // only the two-CTA kernel fuses (see gemm_can_fuse)
   KParams kp{};
   kp.C = a.C;
   kp.Mo = a.Mo;

@@ -104,53 +104,6 @@ __global__ void amax_to_scale_inplace_kernel(uint32_t* bits, int n) {
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Exact division without the per-element IEEE divide sequence.
-//
-// The formats need v = x / S (NVFP4) and t = (x + em) / es (Q4_K) as correctly rounded FP32
-// quotients, because the quotient decides a code. One divisor serves a whole block, so its correctly
-// rounded reciprocal rc = RN(1/y) is computed once and every quotient is then
-//     q0 = RN(x * rc);  q1 = RN(q0 + rc * (x - y*q0))          (x - y*q0 is exact in a fused multiply-add)
-// (two elements per instruction). With an exactly rounded reciprocal and no overflow / underflow in
-// the residual, q1 is the correctly rounded quotient (Markstein's division theorem); the range guard
-// below keeps operands where that holds and the caller falls back to the IEEE divide otherwise.
-// qf_selftest_div compares it with the IEEE divide (tens of billions of pairs, including every BF16
-// numerator and divisors with an all-ones significand, without a difference).
-//
-// The residual is formed rounding toward minus infinity. Being exact, its value does not depend on the
-// rounding mode, but its sign when it is zero does: an exactly cancelling sum is -0 in that mode, so the
-// correction step adds -0 to q0 and leaves q0's sign alone. That makes x = -0 come out as -0, like the
-// IEEE quotient (with round-to-nearest the residual would be +0 and (+0) + (-0) = +0).
-// ---------------------------------------------------------------------------------------------
-
-#ifndef QF_DIV_STEPS
-#define QF_DIV_STEPS 1      // residual corrections after the first product (1 suffices with an exact reciprocal)
-#endif
-
-
-__device__ __forceinline__ float2 div2_fast(float2 x, float y, float rc) {
-  const float2 ny = splat(-y), r = splat(rc);
-  float2 q = __fmul2_rn(x, r);
-  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
-#if QF_DIV_STEPS > 1
-  q = __ffma2_rn(__ffma2_rd(ny, q, x), r, q);
-#endif
-  return q;
-}
-__device__ __forceinline__ float div1_fast(float x, float y, float rc) {
-  float q = __fmul_rn(x, rc);
-  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
-#if QF_DIV_STEPS > 1
-  q = __fmaf_rn(__fmaf_rd(-y, q, x), rc, q);
-#endif
-  return q;
-}
-// divisor magnitudes for which the iteration above is used
-__device__ __forceinline__ bool div_safe(float y) { return y >= 0x1p-60f && y <= 0x1p60f; }
-
-
-
-
 // max |x| over 16 BF16 values held in 8 words, as BF16 bits (sign clear)
 __device__ __forceinline__ uint32_t unit_amax_bits(const uint32_t (&w)[8]) {
   __nv_bfloat162 m0 = __hmax2(__habs2(bits_bf2(w[0])), __habs2(bits_bf2(w[1])));
@@ -239,21 +192,6 @@ __device__ __forceinline__ UnitOut nvfp4_unit(const uint32_t (&w)[8], float amax
 }
 
 constexpr int kUnitsPerThread = 2;
-
-// NVFP4 per-tensor constants derived from the tensor scale: the divisor 6 * s_t of the block-scale quotient and its
-// exactly rounded reciprocal (when the divisor lies in the range where the reciprocal-based division is exact).
-struct Nvfp4Tensor {
-  float s_t, denom, rc_denom;
-  bool denom_safe;
-};
-__device__ __forceinline__ Nvfp4Tensor nvfp4_tensor(float s_t) {
-  Nvfp4Tensor t;
-  t.s_t = s_t;
-  t.denom = __fmul_rn(6.0f, s_t);
-  t.denom_safe = div_safe(t.denom);
-  t.rc_denom = t.denom_safe ? __frcp_rn(t.denom) : 0.0f;
-  return t;
-}
 
 // The grid-stride loop shared by the single-tensor and the batched FP4 kernels: this thread's units are
 // first, first + stride, ... (two in flight per iteration). Every thread of the block must call it (the optional
@@ -949,6 +887,20 @@ cudaError_t launch_qdq_nvfp4_derive(const QdqArgs& a, uint32_t* header, int amax
   }
   q.amax_bits = amax_bits;
   return launch_qdq(q, st);
+}
+
+// Tensor scale(s) alone, for a caller that quantizes the tensor somewhere else (inside the matmul kernel): the maxima,
+// then amax / (6 * 448) into a.tscale_out[0 .. groups-1]. `header` must have been zeroed on the stream beforehand.
+cudaError_t launch_nvfp4_scales_only(const QdqArgs& a, uint32_t* header, int amax_word, cudaStream_t st) {
+  if (a.groups > 1) {
+    uint32_t* bits = reinterpret_cast<uint32_t*>(a.tscale_out);
+    if (cudaError_t e = cudaMemsetAsync(bits, 0, sizeof(uint32_t) * a.groups, st)) return e;
+    if (cudaError_t e = launch_amax_grouped(a.in, a.rows * a.cols / a.groups, a.groups, bits, st)) return e;
+    amax_to_scale_inplace_kernel<<<(a.groups + kThreads - 1) / kThreads, kThreads, 0, st>>>(bits, a.groups);
+    return cudaGetLastError();
+  }
+  if (cudaError_t e = launch_amax(a.in, a.rows * a.cols, header + amax_word, st)) return e;
+  return launch_amax_to_scale(header + amax_word, a.tscale_out, st);
 }
 
 // NVFP4 with a guessed tensor scale in *a.tscale_out (say, the scale of the previous training step). Pass one quantizes

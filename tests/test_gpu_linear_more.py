@@ -177,3 +177,105 @@ def test_forward_with_an_empty_contraction_gives_zeros():
         Y = torch.full((300, 264), float("nan"), dtype=dt, device="cuda")
         api.qf_fq_linear_fwd(X, W, api.FMT_MXFP4, api.FMT_MXFP4, Y=Y)
         assert torch.count_nonzero(Y) == 0
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_MXFP4, api.FMT_MXFP4), (api.FMT_MXFP4, api.FMT_NONE), (api.FMT_NONE, api.FMT_MXFP4)])
+def test_in_kernel_quantization_in_grouped_layers(wq, aq):
+    """QF_FUSED_QDQ in the per-expert calls: ragged, odd-length and empty segments, forward and both backward products,
+    bit for bit the default path, and the default path against the per-expert oracle."""
+    E, H, F = 7, 512, 520
+    offs = _segments([1, 3, 0, 2, 5, 1, 4])
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 61); W = synth.randn_bf16((E, F, H), 0.02, 62); dYp = synth.randn_bf16((rows, F), 1e-3, 63)
+    Xd, Wd, dYd, od = Xp.cuda(), W.cuda(), dYp.cuda(), offs.cuda()
+    ws = api.workspace(api.OP_GROUPED_BWD, rows, F, H, E)
+    y0 = api.qf_fq_grouped_linear_fwd(Xd, Wd, od, wq, aq, y_dtype=torch.float32, ws=ws)
+    dx0, dw0 = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    y1 = api.qf_fq_grouped_linear_fwd(Xd, Wd, od, wq, aq, y_dtype=torch.float32, ws=ws, flags=api.FUSED_QDQ)
+    dx1, dw1 = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws,
+                                            flags=api.FUSED_QDQ)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+    y_ref, dx_ref, dw_ref = _grouped_oracle(Xp, W, dYp, offs, wq, aq)
+    _close(y1, y_ref, "Y"); _close(dx1, dx_ref, "dX"); _close(dw1, dw_ref, "dW")
+
+
+def test_in_kernel_quantization_full_size_moe_gate_up():
+    """The 128-expert gate-and-up projection at full size with the quantizers inside the grouped matmul kernels."""
+    tokens, E, top_k, F, H = 16384, 128, 8, 1536, 2048
+    r = synth.moe_routing(tokens, E, top_k, seed=0)
+    Xp = synth.gather_rows(synth.randn_bf16((tokens, H), 1.0, 1), r.token_of_row).cuda()
+    W = synth.randn_bf16((E, F, H), 0.02, 2, device="cuda")
+    dYp = synth.randn_bf16((Xp.shape[0], F), 1e-3, 3, device="cuda")
+    dYp[(r.token_of_row < 0).cuda()] = 0
+    offs = r.group_offsets.cuda()
+    fmt = api.FMT_MXFP4
+    ws = api.workspace(api.OP_GROUPED_BWD, Xp.shape[0], F, H, E)
+    y0 = api.qf_fq_grouped_linear_fwd(Xp, W, offs, fmt, fmt, ws=ws)
+    dx0, dw0 = api.qf_fq_grouped_linear_bwd(dYp, Xp, W, offs, fmt, fmt, ws=ws)
+    y1 = api.qf_fq_grouped_linear_fwd(Xp, W, offs, fmt, fmt, ws=ws, flags=api.FUSED_QDQ)
+    dx1, dw1 = api.qf_fq_grouped_linear_bwd(dYp, Xp, W, offs, fmt, fmt, ws=ws, flags=api.FUSED_QDQ)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+
+
+@pytest.mark.parametrize("wq,aq", [(api.FMT_NVFP4, api.FMT_NONE), (api.FMT_NVFP4, api.FMT_NVFP4), (api.FMT_MXFP4, api.FMT_NVFP4),
+                                   (api.FMT_NVFP4, api.FMT_MXFP4)])
+@pytest.mark.parametrize("M,N,K", [(520, 776, 1024), (2560, 2304, 832)])
+@pytest.mark.parametrize("given", [False, True])
+def test_in_kernel_nvfp4_quantization_is_bitwise_the_workspace_path(wq, aq, M, N, K, given):
+    """QF_FUSED_QDQ with NVFP4 operands: the tensor scale is settled first (supplied, or derived by a maximum pass
+    over the operand), then the matmul kernel quantizes the staged tiles with the stand-alone quantizer's arithmetic.
+    Same bits as the default path, forward and backward; derived scales are written back all the same."""
+    c = synth.linear_case(M, N, K, seed=M + K + 1, outlier_channels=3, device="cuda")
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    def scales():
+        if not given:
+            return torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda"), 0
+        w_ts = np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.W))["tensor_scale"]) * np.float32(1.25)
+        a_ts = np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(c.X))["tensor_scale"]) * np.float32(0.75)
+        return (torch.tensor([w_ts], device="cuda"), torch.tensor([a_ts], device="cuda"), api.W_TSCALE_GIVEN | api.A_TSCALE_GIVEN)
+    wts0, ats0, fl = scales()
+    y0 = api.qf_fq_linear_fwd(c.X, c.W, wq, aq, y_dtype=torch.float32, ws=ws, w_tscale=wts0, a_tscale=ats0, flags=fl)
+    dx0, dw0 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws,
+                                    w_tscale=wts0, a_tscale=ats0, flags=fl)
+    wts1, ats1, fl = scales()
+    amax = torch.zeros(1, device="cuda")
+    y1 = api.qf_fq_linear_fwd(c.X, c.W, wq, aq, y_dtype=torch.float32, ws=ws, w_tscale=wts1, a_tscale=ats1, a_amax_out=amax,
+                              flags=fl | api.FUSED_QDQ)
+    dx1, dw1 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws,
+                                    w_tscale=wts1, a_tscale=ats1, flags=fl | api.FUSED_QDQ)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(wts0, wts1) and torch.equal(ats0, ats1)
+    assert amax.item() == c.X.abs().max().item()
+    assert torch.equal(y0, y1), "Y"
+    assert torch.equal(dx0, dx1), "dX"
+    assert torch.equal(dw0, dw1), "dW"
+
+
+def test_in_kernel_nvfp4_quantization_in_grouped_layers_with_per_expert_scales():
+    E, H, F = 6, 512, 520
+    offs = _segments([2, 3, 0, 1, 4, 2])
+    rows = int(offs[-1])
+    Xp = synth.randn_bf16((rows, H), 1.0, 71)
+    W = synth.randn_bf16((E, F, H), 0.02, 72)
+    W = (W.float() * torch.tensor([1.0, 4.0, 0.25, 8.0, 0.5, 2.0]).view(E, 1, 1)).to(torch.bfloat16)
+    dYp = synth.randn_bf16((rows, F), 1e-3, 73)
+    Xd, Wd, dYd, od = Xp.cuda(), W.cuda(), dYp.cuda(), offs.cuda()
+    ws = api.workspace(api.OP_GROUPED_BWD, rows, F, H, E)
+    out = []
+    for fl in (0, api.FUSED_QDQ):
+        wts, ats = torch.zeros(E, device="cuda"), torch.zeros(1, device="cuda")
+        y = api.qf_fq_grouped_linear_fwd(Xd, Wd, od, api.FMT_NVFP4, api.FMT_NVFP4, y_dtype=torch.float32, ws=ws, w_tscale=wts,
+                                         a_tscale=ats, flags=fl)
+        dx, dw = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, api.FMT_NVFP4, api.FMT_NVFP4, dx_dtype=torch.float32,
+                                              dw_dtype=torch.float32, ws=ws, w_tscale=wts, a_tscale=ats, flags=fl)
+        assert api.qf_read_status(ws) == 0
+        out.append((y, dx, dw, wts, ats))
+    for a, b in zip(*out):
+        assert torch.equal(a, b)
+    w_ts = [np.float32(oracle.qdq(api.FMT_NVFP4, torch_to_bits(W[g]))["tensor_scale"]) for g in range(E)]
+    assert [np.float32(v) for v in out[1][3].cpu().tolist()] == w_ts
+    a_ts = float(oracle.qdq(api.FMT_NVFP4, torch_to_bits(Xp))["tensor_scale"])
+    y_ref, dx_ref, dw_ref = _grouped_oracle(Xp, W, dYp, offs, api.FMT_NVFP4, api.FMT_NVFP4, w_ts, a_ts)
+    _close(out[1][0], y_ref, "Y"); _close(out[1][1], dx_ref, "dX"); _close(out[1][2], dw_ref, "dW")
