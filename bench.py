@@ -266,15 +266,31 @@ def _graph(torch, fn):
     return g
 
 
-def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
+def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index, which, region_seconds=1.0):
+    """The other named workloads; `which` is a subset of {"cfg1", "cfg3", "cfg4", "cfg5"}; timed regions last at least
+    region_seconds (0: a handful of repetitions, for profiler captures)."""
     out = {}
+    rs = region_seconds
+    wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
     hbm = peaks["hbm_gbs"]
     rate = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
     bw = lambda g: {"gbs": g, "frac_of_measured_hbm": g / hbm, "frac_of_8000_nominal": g / 8000.0}
+    if "cfg1" in which:
+        _cfg1(torch, api, synth, dev, gpu_index, out, bw, rate, wsq, rs)
+    if "cfg3" in which:
+        _cfg3(torch, api, synth, dev, gpu_index, out, bw, rate, wsq, rs)
+    if "cfg4" in which:
+        _cfg4(torch, api, synth, dev, gpu_index, out, peaks, rs)
+    if "cfg5" in which:
+        _cfg5(torch, api, synth, dev, gpu_index, out, peaks, rs)
+    return out
+
+
+def _cfg1(torch, api, synth, dev, gpu_index, out, bw, rate, wsq, rs):
     # ---- 1: NVFP4 QDQ of 2048x2048 weights (all outputs, scale derived from the tensor) -----------------
     mats = [synth.weight_with_outliers(2048, 2048, seed=i, device=dev) for i in range(32)]
     o = torch.empty_like(mats[0]); c = torch.empty((2048, 1024), dtype=torch.uint8, device=dev)
-    sc = torch.empty((2048, 128), dtype=torch.uint8, device=dev); wsq = api.workspace(api.OP_QDQ, 0, 0, 0, device=dev)
+    sc = torch.empty((2048, 128), dtype=torch.uint8, device=dev)
     ts1 = torch.empty(1, dtype=torch.float32, device=dev)
     one = lambda m: api.qf_qdq(api.FMT_NVFP4, m, out=o, codes=c, scales=sc, ws=wsq, tensor_scale=None, ts_out=ts1)
     nbytes = 19136516
@@ -288,10 +304,13 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
                     "pre-pass + quantize), batched = one qf_qdq_batched call for the 32 matrices"}
     for name, g in (("single_cold_l2", g_cold), ("single_warm_l2", g_warm), ("batched_32", g_batch),
                     ("batched_32_speculated_scales_hit", g_spec)):
-        ms, reps, clk = _timed_region(torch, gpu_index, g.replay, min_seconds=0.2)
+        ms, reps, clk = _timed_region(torch, gpu_index, g.replay, min_seconds=0.2 * min(rs, 1.0))
         cfg1[name] = {"us_per_matrix": ms * 1e3 / 32, **bw(rate(32 * nbytes, ms)), "clocks": clk}
     out["nvfp4_qdq_2048x2048"] = cfg1
     del mats, batch, g_cold, g_warm, g_batch, g_spec
+
+
+def _cfg3(torch, api, synth, dev, gpu_index, out, bw, rate, wsq, rs):
     # ---- 3: Q4_K QDQ over all linear weights of the 32-layer dense decoder, per-layer seeds (14 GB of weights
     # resident; outputs go to one layer's buffers, reused) ------------------------------------------------------
     layers = [[synth.dense_decoder_weight(l, name, device=dev) for name, _, _ in synth.DENSE_DECODER_LAYER]
@@ -305,12 +324,15 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
             for w, oo, cc, ss in zip(layer, outs, codes, scs):
                 api.qf_qdq(api.FMT_Q4_K, w, out=oo, codes=cc, scales=ss, ws=wsq)
     g3 = _graph(torch, q4k_all)
-    ms, reps, clk = _timed_region(torch, gpu_index, g3.replay, min_seconds=0.5, warm=1, probe=2)
+    ms, reps, clk = _timed_region(torch, gpu_index, g3.replay, min_seconds=0.5 * min(rs, 1.0), warm=1, probe=2)
     elems = synth.dense_decoder_layer_elems() * synth.DENSE_DECODER_LAYERS
     out["q4k_qdq_dense_decoder_32_layers"] = {"ms": ms, "elements": elems, **bw(rate(elems * 4.5625, ms)), "reps": reps, "clocks": clk,
                                               "note": "224 distinct weight tensors (per-layer seeds), one qf_qdq call each, as one CUDA graph"}
     del layers, outs, codes, scs, g3
     torch.cuda.empty_cache()
+
+
+def _cfg4(torch, api, synth, dev, gpu_index, out, peaks, rs):
     # ---- 4: NVFP4 weight-only linear, one 32K-token sequence, up and down projections, fwd + bwd ---------------
     Mt = 32768
     tot_ms, tot_fl, parts = 0.0, 0.0, {}
@@ -323,7 +345,7 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
         def f4():
             api.qf_fq_linear_fwd(cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, Y=Y, w_tscale=wts)
             api.qf_fq_linear_bwd(cse.dY, cse.X, cse.W, api.FMT_NVFP4, api.FMT_NONE, ws=ws4, dX=dX, dW=dW, w_tscale=wts)
-        ms, reps, clk = _timed_region(torch, gpu_index, f4, min_seconds=1.0, warm=2, probe=2)
+        ms, reps, clk = _timed_region(torch, gpu_index, f4, min_seconds=rs, warm=2, probe=2)
         fl = 3 * 2.0 * Mt * Nn * Kk
         parts[pname] = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "reps": reps, "clocks": clk}
         tot_ms += ms; tot_fl += fl
@@ -332,6 +354,9 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
     out["nvfp4_weight_only_linear_32k_tokens_up_down"] = {"ms": tot_ms, "tflops": t4, "frac_of_2250_datasheet": t4 / DATASHEET_TFLOPS,
                                                            "frac_of_measured_sustained": t4 / peaks["bf16_sustained"],
                                                            "frac_of_measured_burst": t4 / peaks["bf16_burst"], **parts}
+
+
+def _cfg5(torch, api, synth, dev, gpu_index, out, peaks, rs):
     # ---- 5: MoE grouped MXFP4 W4A4: 128 experts, top-8 of 16384 tokens, gate + up + down, fwd + bwd. The gate and up
     # projections are stored as one [E, 2F, H] weight, as serving engines keep them: the same products (the quantizer's
     # blocks run along H, so quantizing the concatenation is concatenating the quantized halves), and the routed
@@ -354,7 +379,7 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
             api.qf_fq_grouped_linear_fwd(Xp, Wg, offs, fmt, fmt, ws=ws5, Y=Y)
             api.qf_fq_grouped_linear_bwd(dYp, Xp, Wg, offs, fmt, fmt, ws=ws5, dX=dX, dW=dw, flags=flags)
         for key, fn in (("default", f5), ("reuse", lambda: f5(flags=api.REUSE_W_HAT | api.REUSE_X_HAT)), ("bf16_dw", lambda: f5(dw=dW16))):
-            ms, reps, clk = _timed_region(torch, gpu_index, fn, min_seconds=1.0 if key == "default" else 0.3)
+            ms, reps, clk = _timed_region(torch, gpu_index, fn, min_seconds=rs if key == "default" else 0.3 * min(rs, 1.0))
             res[key][0] += ms
             res[key][1] = clk
         del Xp, Wg, dYp, ws5, Y, dX, dW, dW16
@@ -367,7 +392,6 @@ def measure_other_workloads(torch, api, synth, dev, peaks, gpu_index):
         "layout": "gate and up as one [128, 1536, 2048] grouped weight, down [128, 2048, 768]; dW in FP32",
         "ms_reusing_forward_copies": res["reuse"][0], "tflops_reusing_forward_copies": tf(res["reuse"][0]),
         "ms_with_bf16_dw": res["bf16_dw"][0], "tflops_with_bf16_dw": tf(res["bf16_dw"][0])}
-    return out
 
 
 # -------------------------------------------------------------------------------------------------
@@ -600,10 +624,11 @@ def run_ours(args):
                          f"included, {dt:.1f} s"}
 
     other = None
-    if rank == 0 and world == 1 and "configs" in sections:
+    which = {"cfg1", "cfg3", "cfg4", "cfg5"} if "configs" in sections else sections & {"cfg1", "cfg3", "cfg4", "cfg5"}
+    if rank == 0 and world == 1 and which:
         del X, W, dY, Y, dX, dW, ws
         torch.cuda.empty_cache()
-        other = measure_other_workloads(torch, api, synth, dev, peaks, gpu_index)
+        other = measure_other_workloads(torch, api, synth, dev, peaks, gpu_index, which, args.region_seconds)
 
     if rank == 0:
         clocks = clk.summary()
@@ -653,7 +678,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sections", default=",".join(SECTIONS),
                     help="measurements beside the headline: roofline, sustained, qdq, e2e, cpu, configs (the other named "
-                         "workloads); all by default (empty string: none)")
+                         "workloads; cfg1 / cfg3 / cfg4 / cfg5 pick single ones); all by default (empty string: none)")
+    ap.add_argument("--region-seconds", type=float, default=1.0,
+                    help="minimum length of the timed regions of the other named workloads (0 for profiler captures)")
     ap.add_argument("--shape", default=None, help="M,N,K of a smaller case (profiler captures only)")
     ap.add_argument("--in-kernel-qdq", action="store_true",
                     help="run the step with QF_FUSED_QDQ (quantize the staged tiles inside the matmul kernel) instead of the default path")
