@@ -6,8 +6,8 @@
 One step = one pass of the whole path over one batch: the quantization-aware linear layer with
 MXFP4 weights and activations, forward plus straight-through backward (dX and dW), on
 X [8192,4096], W [12288,4096], dY [8192,12288] — i.e. two quantize-dequantize passes over W and X
-(forward, and again in the backward, since the fake-quantized copies are transient) and three BF16
-tensor-core matmuls. Prints ONE JSON line (rank 0). Multi-GPU runs are independent replicas of
+(forward, and again in the backward, since the fake-quantized copies are transient; the backward's pass over X
+rides inside the dX matmul launch) and three BF16 tensor-core matmuls. Prints ONE JSON line (rank 0). Multi-GPU runs are independent replicas of
 the same workload (the path has no exchange step): weak scaling, no data-path collective. With
 ``--gpus N`` (N > 1) and no torchrun environment the script starts the N ranks itself.
 
@@ -50,7 +50,7 @@ def _set_shape(spec: str):
     WORKLOAD = f"mxfp4_w4a4_linear_fwd_bwd_{M}x{K}x{N}"
     FLOP_PER_GEMM = 2.0 * M * N * K
     FLOP_PER_STEP = 3.0 * FLOP_PER_GEMM
-KERNELS_PER_STEP = 7          # fwd: qdq(W), qdq(X), gemm; bwd: qdq(W), gemm, qdq(X), gemm
+KERNELS_PER_STEP = 6          # fwd: qdq(W), qdq(X), gemm; bwd: qdq(W), gemm (dX, with qdq(X) as its side job), gemm (dW)
 
 
 def _peaks():

@@ -217,6 +217,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
   }
   Workspace w = carve(ws, N, K, groups);
   if (cudaError_t e = cudaMemsetAsync(w.header, 0, kWsHeader, st)) return cu(e);
+  bool x_hat_done = false;          // X_hat already produced by a side job of the dX launch
   if (dX) {
     // dX[M,K] = dY[M,N] . W_hat[N,K]: A = dY contraction-major, B = W_hat stored [contraction N, K]
     GemmArgs g{};
@@ -241,6 +242,18 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
       Wh = w.w_hat;
     }
     g.B = Wh;
+    // The activations' quantize pass belongs to the next product (dW). It is HBM-bound and this product is tensor-bound,
+    // so where the kernel can carry it (MXFP4, or NVFP4 with a supplied scale) it runs as a side job of this launch.
+    if (dW && (aq == QF_FMT_MXFP4 || (aq == QF_FMT_NVFP4 && (flags & QF_A_TSCALE_GIVEN))) && !(flags & (QF_REUSE_X_HAT | QF_FUSED_QDQ)) &&
+        M * K > 0 && (M * K) % 32 == 0 && gemm_side_supported(g)) {
+      g.side[0].in = X;
+      g.side[0].out = w.x_hat;
+      g.side[0].nelem = M * K;
+      g.side[0].fmt = aq;
+      g.side[0].tscale = a_ts;
+      g.side[0].mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
+      x_hat_done = true;
+    }
     if (cudaError_t e = launch_gemm(g, st)) return cu(e);
   }
   if (dW) {
@@ -262,7 +275,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
       if (aq == QF_FMT_NVFP4)
         if (qf_status_t s = fused_nvfp4_scale(X, M, K, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, 1, st, &g.fuse_b_tscale)) return s;
     } else if (aq != QF_FMT_NONE) {
-      if (!(flags & QF_REUSE_X_HAT))
+      if (!(flags & QF_REUSE_X_HAT) && !x_hat_done)
         if (qf_status_t s = quantize_operand(aq, X, M, K, w.x_hat, a_ts, flags & QF_A_TSCALE_GIVEN, w.header, kWsAmaxA, kWsScaleA, st, 1, (flags & QF_MXFP4_NO_CLIP) != 0)) return s;
       Xh = w.x_hat;
     }

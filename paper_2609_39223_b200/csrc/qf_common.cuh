@@ -309,7 +309,18 @@ struct GemmArgs {
   const float* fuse_b_tscale;        // NVFP4: device tensor scale(s) of B: one float, or one per group (mode 1)
   bool fuse_b_tscale_per_group;
   bool mxfp4_noclip;                 // scale rule of the in-kernel MXFP4 quantizer (QF_MXFP4_NO_CLIP)
+  // Side jobs: flat FP4 quantize-dequantize passes (BF16 copy only) that spare warps of the matmul kernel run while the
+  // tensor cores work, for operands of the NEXT product. Nothing in this launch reads what they write.
+  struct Side {
+    const void* in;                  // BF16, nelem elements (a multiple of 32)
+    void* out;
+    int64_t nelem;                   // 0: no job
+    int fmt;                         // QF_FMT_MXFP4, or QF_FMT_NVFP4 with a final tensor scale at *tscale
+    const float* tscale;
+    bool mxfp4_noclip;
+  } side[2];
 };
+bool gemm_side_supported(const GemmArgs& a);
 
 cudaError_t launch_pack_q4k(const void* codes, const void* scales, int64_t nsb, void* records, bool unpack, void* codes_out,
                             void* scales_out, cudaStream_t st);

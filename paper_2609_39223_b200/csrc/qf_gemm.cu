@@ -23,6 +23,7 @@
 
 #include "qf_common.cuh"
 #include "qf_ptx.cuh"
+#include "qf_qdq_body.cuh"
 
 namespace qf {
 namespace {
@@ -70,6 +71,13 @@ struct KParams {
   const float* a_tscale;             // NVFP4 in-kernel quantizer: tensor scale of A
   const float* b_tscale;             // ... of B: one value, or one per group (grouped mode 1)
   int b_tscale_per_group;
+  struct Side {                      // side jobs of the SIDE variant (see GemmArgs::Side)
+    const uint4* in;
+    uint4* out;
+    int64_t nunits;                  // 16-element units
+    const float* tscale;
+    int fmt, noclip;
+  } side[2];
 };
 
 // ---- descriptors ------------------------------------------------------------------------------
@@ -484,6 +492,8 @@ constexpr int TRANSFORM_WARPS = 16;                      // fused variant: warps
 constexpr int TRANSFORM_GROUPS = 4;                      // group g takes k-blocks g, g + 4, ... (must not exceed STAGES2)
 constexpr int WARPS_PER_GROUP = TRANSFORM_WARPS / TRANSFORM_GROUPS;
 constexpr int NUM_THREADS_FUSED = NUM_THREADS + 32 * TRANSFORM_WARPS;
+constexpr int SIDE_WARPS = 8;                           // SIDE variant: warps that run the side jobs
+constexpr int NUM_THREADS_SIDE = NUM_THREADS + 32 * SIDE_WARPS;
 static_assert(TRANSFORM_GROUPS <= 6, "more groups than pipeline stages would let a group wait on a stage two uses ahead");
 
 struct alignas(8) Barriers2 {
@@ -707,8 +717,10 @@ __device__ __forceinline__ void nvfp4_transform_tile(uint32_t base, int warp_in_
 // TRANSFORM_WARPS extra warps (sixteen, in four groups that take alternate k-blocks) transform each stage in
 // shared memory between the TMA arrival and the MMA issue, so the fake-quantized operand never exists in
 // global memory.
-template <bool A_MN, bool B_MN, typename OutT, int FUSE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FUSE ? NUM_THREADS_FUSED : NUM_THREADS, 1)
+// SIDE: eight more warps run up to two flat FP4 quantize-dequantize passes over other tensors (the operand of the next
+// product) from global to global memory while the tensor cores work: an HBM-bound pass hidden under a tensor-bound one.
+template <bool A_MN, bool B_MN, typename OutT, int FUSE, bool SIDE = false>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FUSE ? NUM_THREADS_FUSED : (SIDE ? NUM_THREADS_SIDE : NUM_THREADS), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -887,6 +899,21 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) mbar_arrive_remote(mapa_shared(smem_u32(&bars->ready[stage]), 0));
       }
     }
+  } else if (SIDE && warp >= 6) {
+    // ===== side jobs (both CTAs): grid-stride over the units of each job; no synchronisation with the other roles =====
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * (32 * SIDE_WARPS) + (threadIdx.x - NUM_THREADS);
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * (32 * SIDE_WARPS);
+#pragma unroll 1
+    for (int j = 0; j < 2; ++j) {
+      const auto& job = p.side[j];
+      if (job.nunits <= 0) continue;
+      if (job.fmt == QF_FMT_NVFP4)
+        qdq_fp4_body<QF_FMT_NVFP4, PlainLoader, false>(PlainLoader{job.in}, job.nunits, job.out, nullptr, nullptr,
+                                                       nvfp4_tensor(__ldg(job.tscale)), false, false, nullptr, first, stride);
+      else
+        qdq_fp4_body<QF_FMT_MXFP4, PlainLoader, false>(PlainLoader{job.in}, job.nunits, job.out, nullptr, nullptr,
+                                                       nvfp4_tensor(1.0f), false, job.noclip != 0, nullptr, first, stride);
+    }
   } else {
     // ===== epilogue (both CTAs): own 128 accumulator rows =====
     const int quarter = warp & 3;
@@ -1039,10 +1066,10 @@ cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUten
   return cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN, typename OutT, int FUSE>
+template <bool A_MN, bool B_MN, typename OutT, int FUSE, bool SIDE = false>
 cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const KParams& kp, int grid,
                           cudaStream_t st) {
-  auto kern = gemm_pair_kernel<A_MN, B_MN, OutT, FUSE>;
+  auto kern = gemm_pair_kernel<A_MN, B_MN, OutT, FUSE, SIDE>;
   static bool configured[64] = {false};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
@@ -1051,7 +1078,7 @@ cudaError_t launch_pair_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const 
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  kern<<<grid, FUSE ? NUM_THREADS_FUSED : NUM_THREADS, SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);   // cluster shape (2,1,1) is a kernel attribute
+  kern<<<grid, FUSE ? NUM_THREADS_FUSED : (SIDE ? NUM_THREADS_SIDE : NUM_THREADS), SMEM2_BYTES, st>>>(tmA, tmB, tmC, kp);   // cluster shape (2,1,1) is a kernel attribute
   return cudaGetLastError();
 }
 
@@ -1059,6 +1086,11 @@ template <typename OutT>
 cudaError_t launch_pair_majors(const GemmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
                                const KParams& kp, int grid, cudaStream_t st) {
   const int fuse = (a.fuse_a_fmt ? 1 : 0) | (a.fuse_b_fmt ? 2 : 0);
+  if (a.side[0].nelem > 0 || a.side[1].nelem > 0) {
+    if (fuse != 0 || a.a_mn_major) return cudaErrorInvalidValue;          // see gemm_side_supported
+    if (a.b_mn_major) return launch_pair_t<false, true, OutT, 0, true>(tmA, tmB, tmC, kp, grid, st);
+    return launch_pair_t<false, false, OutT, 0, true>(tmA, tmB, tmC, kp, grid, st);
+  }
   if (!a.a_mn_major && !a.b_mn_major) {
     if (fuse == 3) return launch_pair_t<false, false, OutT, 3>(tmA, tmB, tmC, kp, grid, st);
     if (fuse == 2) return launch_pair_t<false, false, OutT, 2>(tmA, tmB, tmC, kp, grid, st);
@@ -1112,6 +1144,14 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.a_tscale = a.fuse_a_tscale;
   kp.b_tscale = a.fuse_b_tscale;
   kp.b_tscale_per_group = a.fuse_b_tscale_per_group ? 1 : 0;
+  for (int j = 0; j < 2; ++j) {
+    kp.side[j].in = static_cast<const uint4*>(a.side[j].in);
+    kp.side[j].out = static_cast<uint4*>(a.side[j].out);
+    kp.side[j].nunits = a.side[j].nelem / 16;
+    kp.side[j].tscale = a.side[j].tscale;
+    kp.side[j].fmt = a.side[j].fmt;
+    kp.side[j].noclip = a.side[j].mxfp4_noclip ? 1 : 0;
+  }
   kp.group_mode = a.group_mode;
   kp.G = a.G;
   kp.offs = a.group_offsets;
@@ -1162,10 +1202,14 @@ static bool pair_applies(const GemmArgs& a) {
 // (plain and grouped problems alike: the transform works on whatever tile the producer staged).
 bool gemm_can_fuse(const GemmArgs& a) { return pair_applies(a); }
 
+// True if this product runs on the two-CTA kernel in a variant that can carry side jobs (forward and dX products
+// without the in-kernel quantizer). A launch with side jobs always uses every SM, however few tiles it has.
+bool gemm_side_supported(const GemmArgs& a) { return pair_applies(a) && !a.a_mn_major && !a.fuse_a_fmt && !a.fuse_b_fmt; }
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0) return cudaSuccess;
   if (pair_applies(a)) return launch_gemm_pair(a, st);
-  if (a.fuse_a_fmt || a.fuse_b_fmt) return cudaErrorInvalidValue;           // only the two-CTA kernel fuses (see gemm_can_fuse)
+  if (a.fuse_a_fmt || a.fuse_b_fmt || a.side[0].nelem > 0 || a.side[1].nelem > 0) return cudaErrorInvalidValue;   // only the two-CTA kernel fuses or carries side jobs
   KParams kp{};
   kp.C = a.C;
   kp.Mo = a.Mo;
