@@ -279,3 +279,37 @@ def test_in_kernel_nvfp4_quantization_in_grouped_layers_with_per_expert_scales()
     a_ts = float(oracle.qdq(api.FMT_NVFP4, torch_to_bits(Xp))["tensor_scale"])
     y_ref, dx_ref, dw_ref = _grouped_oracle(Xp, W, dYp, offs, api.FMT_NVFP4, api.FMT_NVFP4, w_ts, a_ts)
     _close(out[1][0], y_ref, "Y"); _close(out[1][1], dx_ref, "dX"); _close(out[1][2], dw_ref, "dW")
+
+
+@pytest.mark.parametrize("aq,given", [(api.FMT_MXFP4, False), (api.FMT_NVFP4, True)])
+@pytest.mark.parametrize("M,N,K", [(520, 776, 1024), (2560, 2304, 832), (257, 264, 96)])
+def test_backward_with_the_activation_pass_inside_the_dx_launch_is_bitwise_the_two_separate_products(aq, given, M, N, K):
+    """A backward call that asks for both gradients lets spare warps of the dX launch quantize X for the dW product.
+    The gradients must be the bits that two separate calls (dX alone, dW alone: no side job) produce."""
+    c = synth.linear_case(M, N, K, seed=M + 3 * K, outlier_channels=2, device="cuda")
+    wq = api.FMT_MXFP4
+    ws = api.workspace(api.OP_LINEAR_BWD, M, N, K)
+    ats = torch.tensor([0.01], device="cuda") if given else None
+    fl = api.A_TSCALE_GIVEN if given else 0
+    dx0, _ = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, want_dw=False, ws=ws, a_tscale=ats, flags=fl)
+    _, dw0 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dw_dtype=torch.float32, want_dx=False, ws=ws, a_tscale=ats, flags=fl)
+    ws.zero_()                                    # nothing may be left over from the separate calls
+    dx1, dw1 = api.qf_fq_linear_bwd(c.dY, c.X, c.W, wq, aq, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws, a_tscale=ats, flags=fl)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+
+
+def test_grouped_backward_with_the_activation_pass_inside_the_dx_launch():
+    E, H, F = 7, 512, 520
+    offs = _segments([1, 3, 0, 2, 5, 1, 4])
+    rows = int(offs[-1])
+    Xd = synth.randn_bf16((rows, H), 1.0, 81, device="cuda"); Wd = synth.randn_bf16((E, F, H), 0.02, 82, device="cuda")
+    dYd = synth.randn_bf16((rows, F), 1e-3, 83, device="cuda"); od = offs.cuda()
+    fmt = api.FMT_MXFP4
+    ws = api.workspace(api.OP_GROUPED_BWD, rows, F, H, E)
+    dx0, _ = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, fmt, fmt, dx_dtype=torch.float32, want_dw=False, ws=ws)
+    _, dw0 = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, fmt, fmt, dw_dtype=torch.float32, want_dx=False, ws=ws)
+    ws.zero_()
+    dx1, dw1 = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
+    assert api.qf_read_status(ws) == 0
+    assert torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
