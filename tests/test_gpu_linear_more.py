@@ -313,3 +313,24 @@ def test_grouped_backward_with_the_activation_pass_inside_the_dx_launch():
     dx1, dw1 = api.qf_fq_grouped_linear_bwd(dYd, Xd, Wd, od, fmt, fmt, dx_dtype=torch.float32, dw_dtype=torch.float32, ws=ws)
     assert api.qf_read_status(ws) == 0
     assert torch.equal(dx0, dx1) and torch.equal(dw0, dw1)
+
+
+def test_weight_gradient_with_a_contraction_cut_into_chunks():
+    """At 32768 tokens and more an FP32 dW is computed in chunks of 16384 tokens, the later launches adding into the
+    first one's result. 40000 tokens give chunks of 16384 + 16384 + 7232 rows; with and without the caller's own
+    accumulation flag, against the oracle."""
+    M, N, K = 40000, 264, 96
+    c = synth.linear_case(M, N, K, seed=77, outlier_channels=1)
+    fmt = api.FMT_MXFP4
+    _, dw_ref = oracle.fq_linear_bwd(torch_to_bits(c.dY), torch_to_bits(c.X), torch_to_bits(c.W), fmt, fmt)
+    X, W, dY = c.X.cuda(), c.W.cuda(), c.dY.cuda()
+    dw = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
+    api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, want_dx=False, dW=dw)
+    _close(dw, dw_ref, "dW")
+    base = torch.randn((N, K), device="cuda") * 1e-2
+    acc = base.clone()
+    api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, want_dx=False, dW=acc, flags=api.ACCUMULATE_DW)
+    _close(acc - base, dw_ref, "dW accumulated")
+    dw16 = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")           # BF16 output: one launch, no chunks
+    api.qf_fq_linear_bwd(dY, X, W, fmt, fmt, want_dx=False, dW=dw16)
+    assert (dw16.float() - dw).abs().max().item() <= dw.abs().max().item() * 2.0 ** -8
