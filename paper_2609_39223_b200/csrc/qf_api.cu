@@ -194,6 +194,7 @@ qf_status_t linear_fwd_impl(const void* X, const void* W, void* Y, int y_dtype, 
   if (a_amax_out)
     if (cudaError_t e = launch_amax_to_float(amax_word, a_amax_out, st)) return cu(e);
   g.A = Xh; g.B = Wh;
+  g.tile_sync_word = w.header + kWsTileSync;
   return cu(launch_gemm(g, st));
 }
 
@@ -256,6 +257,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
       g.side[0].mxfp4_noclip = (flags & QF_MXFP4_NO_CLIP) != 0;
       x_hat_done = true;
     }
+    g.tile_sync_word = w.header + kWsTileSync;
     if (cudaError_t e = launch_gemm(g, st)) return cu(e);
   }
   if (dW) {
@@ -290,6 +292,7 @@ qf_status_t linear_bwd_impl(const void* dY, const void* X, const void* W, void* 
     for (int64_t c = 0; c < chunks; ++c) {
       const int64_t r0 = c * kWgradChunkRows;
       GemmArgs gc = g;
+      gc.tile_sync_word = c + 1 < kWsTileSyncCount ? w.header + kWsTileSync + 1 + c : nullptr;
       if (chunks > 1) {
         gc.A = static_cast<const uint8_t*>(g.A) + static_cast<size_t>(r0) * N * 2;
         gc.B = static_cast<const uint8_t*>(g.B) + static_cast<size_t>(r0) * K * 2;

@@ -26,6 +26,8 @@ enum WsWord : int {
   kWsGuessW = 10,     // the caller's guess of W's tensor scale (float bits), kept for the conditional second pass
   kWsClkCycles = 12,  // 64-bit: SM clock cycles the last matmul launch ran for (first CTA, start to end)
   kWsClkNanos = 14,   // 64-bit: the same interval in nanoseconds of the global timer; cycles / ns = SM clock in GHz
+  kWsTileSync = 24,   // 16 words: arrival counters of the matmul launches of one call (tile-start rendezvous)
+  kWsTileSyncCount = 16,
 };
 
 // ---- device helpers -----------------------------------------------------------------------
@@ -303,6 +305,7 @@ struct GemmArgs {
   int64_t c_group_stride;        // elements between consecutive groups of C (mode 2)
   int64_t rows_padded;           // mode 1: total rows of A / C; mode 2: total contraction rows
   uint32_t* status_word;         // device word receiving QF_ERR_TIMEOUT if a wait expires
+  uint32_t* tile_sync_word;      // device word, zero before the launch: arrival counter of the tile-start rendezvous (nullable)
   int fuse_a_fmt, fuse_b_fmt;        // QF_FMT_MXFP4 / QF_FMT_NVFP4: quantize-dequantize the staged tiles of that operand
                                      // inside the kernel (QF_FMT_NONE: the operand is used as it is)
   const float* fuse_a_tscale;        // NVFP4: device tensor scale of A (one float), final before the launch

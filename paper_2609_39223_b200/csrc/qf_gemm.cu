@@ -66,6 +66,8 @@ struct KParams {
   int64_t b_group_rows;      // mode 1: rows one group occupies in B's 2-D tensor map
   int64_t c_group_stride;    // mode 2: elements between per-group outputs
   uint32_t* status;
+  uint32_t* tile_sync;       // plain problems: global arrival counter that keeps the CTA pairs' tile starts together (nullable)
+  long long tile_sync_limit; // SM clocks a pair waits for the others at a tile start before it goes on alone
   int mxfp4_noclip;          // scale rule of the in-kernel MXFP4 quantizer
   int fuse_a_fmt, fuse_b_fmt;        // format of the in-kernel quantizer per operand (QF_FMT_MXFP4 / QF_FMT_NVFP4)
   const float* a_tscale;             // NVFP4 in-kernel quantizer: tensor scale of A
@@ -532,6 +534,11 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster)
       : "memory");
 }
+__device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -794,10 +801,29 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued = 0;
       bool alive = true;
-      for (int t = cluster_id; t < num_tiles && alive; t += num_clusters) {
+      uint32_t local = 0, sync_misses = 0;
+      for (int t = cluster_id; t < num_tiles && alive; t += num_clusters, ++local) {
         const PairTile tile = decode_pair(p, cum, tiles_m, t);
         const int m0 = tile.m0 + static_cast<int>(rank) * BM;
         const int n0 = tile.n0 + static_cast<int>(rank) * (BN / 2);
+        if (p.tile_sync) {
+          // Rendezvous of all CTA pairs at the start of their local-th tile. Pairs that share an operand panel only find
+          // each other's loads in L2 while they walk the contraction together; left alone they drift apart by a few
+          // percent per tile (measured: 2.5 us per 80 us tile) and the sharing is gone after a few waves. Best effort:
+          // a pair waits a fraction of a tile time at most, then goes on alone; after two such misses it stops waiting
+          // (the grid may not be co-resident, e.g. next to another stream's kernel), so nothing can hang or fail.
+          if (leader) atomicAdd(p.tile_sync, 1u);
+          if (local > 0 && sync_misses < 2) {
+            const uint32_t target = static_cast<uint32_t>(min(static_cast<long long>(local + 1) * num_clusters, static_cast<long long>(num_tiles)));
+            const long long t0 = clock64();
+            bool met = true;
+            while (ld_acquire_gpu_u32(p.tile_sync) < target) {
+              if (clock64() - t0 > p.tile_sync_limit) { met = false; break; }
+              __nanosleep(64);
+            }
+            sync_misses = met ? 0u : sync_misses + 1u;
+          }
+        }
         for (int k = tile.k_begin; k < tile.k_end; k += BK) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, p.status)) { alive = false; break; }
           const uint32_t full_local = smem_u32(&bars->full[stage]);
@@ -1138,6 +1164,10 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t st) {
   kp.c_dtype = a.c_dtype;
   kp.accumulate = a.accumulate ? 1 : 0;
   kp.status = a.status_word;
+  // Tile-start rendezvous for plain problems with long contractions (measured at 32768 x 4096 x 14336: DRAM reads of the dX
+  // launch 8.7 -> 4.1 GB, 2719 -> 2480 us; neutral from 8192 to 12288; a loss below, where a tile lasts 25 us).
+  kp.tile_sync = (a.group_mode == 0 && a.Kc >= 8192) ? a.tile_sync_word : nullptr;
+  kp.tile_sync_limit = a.Kc;                   // one eighth of a tile's main loop (Kc / 64 k-blocks of about 512 clocks)
   kp.mxfp4_noclip = a.mxfp4_noclip ? 1 : 0;
   kp.fuse_a_fmt = a.fuse_a_fmt;
   kp.fuse_b_fmt = a.fuse_b_fmt;
