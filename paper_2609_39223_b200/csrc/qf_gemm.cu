@@ -223,9 +223,6 @@ __device__ __forceinline__ void store_chunk32<float>(float* row_ptr, int col0, i
 // accumulating in FP32) of the 32-row box. The tensor map clips rows and columns past the matrix edge.
 // Two staging buffers per warp let the next chunk be converted while the previous store drains.
 
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
@@ -628,12 +625,6 @@ __device__ __forceinline__ PairTile decode_pair(const KParams& p, const int* cum
     r.z = g;
   }
   return r;
-}
-
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-  return v;
 }
 
 // In-place MXFP4 quantize-dequantize of `nchunks` 16-byte chunks of a staged operand tile by the 256

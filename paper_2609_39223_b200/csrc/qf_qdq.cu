@@ -9,6 +9,7 @@
 // operation that decides a code is written with an explicit round-to-nearest intrinsic so that
 // the compiler can neither contract it into an FMA nor replace a division by a reciprocal.
 #include "qf_common.cuh"
+#include "qf_ptx.cuh"
 #include "qf_qdq_body.cuh"
 
 namespace qf {
@@ -232,11 +233,62 @@ constexpr float kRound = 12582912.0f;      // 1.5 * 2^23: adding it rounds to th
 template <bool FAST>
 __device__ __forceinline__ float div_by(float x, float y, float rc) { return FAST ? div1_fast(x, y, rc) : __fdiv_rn(x, y); }
 
-template <bool FAST>
-__device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, float hi, uint4* __restrict__ out_ptr,
-                                             uint32_t (&cbytes)[8], __half& d_h, __half& dmin_h, uint32_t& s6, uint32_t& m6) {
+// Where the four 16-byte groups of a sub-block's dequantized values go: straight to global memory, or into a
+// shared-memory staging tile (slot c of the lane holds chunk c ^ perm, see the staged kernel).
+struct GlobalSink {
+  uint4* out_ptr;                          // nullable: no dequantized copy wanted
+  __device__ __forceinline__ void put(int c, uint4 v) const { if (out_ptr) out_ptr[c] = v; }
+};
+struct SmemSink {
+  uint32_t base;                           // shared address of this lane's 64-byte record
+  uint32_t perm;
+  bool on;
+  __device__ __forceinline__ void put(int c, uint4 v) const {
+    if (on) st_shared_v4(base + ((static_cast<uint32_t>(c) ^ perm) << 4), v.x, v.y, v.z, v.w);
+  }
+};
+
+// The 32 elements of one sub-block given its effective scale and offset: codes (one per byte in cbytes) and dequantized
+// values. CLAMP = false leaves out the clamp of the quotient to [0, 15]: the caller has checked that no quotient of the
+// sub-block can round outside that range.
+template <bool FAST, bool CLAMP, typename Sink>
+__device__ __forceinline__ void q4k_elements(const uint32_t (&w)[16], float es, float em, float rc, bool live, const Sink sink,
+                                             uint32_t (&cbytes)[8]) {
   uint32_t xhat[4];
-  lo = fminf(lo, 0.0f);
+  const float2 em2 = splat(em), nem2 = splat(-em), es2 = splat(es), magic = splat(kRound), nmagic = splat(-kRound);
+  uint32_t ybits[2][2];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float2 x = unpack2(w[j]);
+    float2 y = magic;                                // code 0 when the sub-block has no scale
+    if (FAST || live) {                              // FAST: rc = 0 makes the reciprocal-based quotient 0, no branch needed
+      const float2 num = __fadd2_rn(x, em2);
+      float2 t = FAST ? div2_fast(num, es, rc) : make_float2(__fdiv_rn(num.x, es), __fdiv_rn(num.y, es));
+      if (CLAMP) {
+        t.x = fminf(fmaxf(t.x, 0.0f), 15.0f);        // clamp first: rounding is monotone and 0, 15 are integers
+        t.y = fminf(fmaxf(t.y, 0.0f), 15.0f);
+      }
+      y = __fadd2_rn(t, magic);                      // integer code now sits in the low mantissa bits
+    }
+    const float2 c = __fadd2_rn(y, nmagic);
+    const float2 o = __ffma2_rn(es2, c, nem2);        // product exact: one rounding, as es*c - em
+    xhat[j & 3] = pack_bf16x2(o.x, o.y);
+    if ((j & 3) == 3) sink.put(j >> 2, make_uint4(xhat[0], xhat[1], xhat[2], xhat[3]));               // stored as soon as complete
+    // the low byte of y's bit pattern is the code (the low byte of the rounding constant is zero)
+    ybits[j & 1][0] = __float_as_uint(y.x);
+    ybits[j & 1][1] = __float_as_uint(y.y);
+    if (j & 1) {
+      const uint32_t p01 = __byte_perm(ybits[0][0], ybits[0][1], 0x0040);
+      const uint32_t p23 = __byte_perm(ybits[1][0], ybits[1][1], 0x0040);
+      cbytes[j >> 1] = __byte_perm(p01, p23, 0x5410);             // codes 4k..4k+3, one per byte
+    }
+  }
+}
+
+template <bool FAST, typename Sink>
+__device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo_raw, float hi, const Sink sink,
+                                             uint32_t (&cbytes)[8], __half& d_h, __half& dmin_h, uint32_t& s6, uint32_t& m6) {
+  const float lo = fminf(lo_raw, 0.0f);
   const float sc = div_by<FAST>(__fsub_rn(hi, lo), 15.0f, kRcp15);
   const float off = __fsub_rn(0.0f, lo);            // >= +0: a sub-block with no negative value has offset +0
   float max_sc = sc, max_off = off;
@@ -256,30 +308,91 @@ __device__ __forceinline__ void q4k_subblock(const uint32_t (&w)[16], float lo, 
   const float es = __fmul_rn(d, s6f), em = __fmul_rn(dmin, m6f);
   const bool live = es > 0.0f;
   const float rc = live ? __frcp_rn(es) : 0.0f;
-  const float2 em2 = splat(em), nem2 = splat(-em), es2 = splat(es), magic = splat(kRound), nmagic = splat(-kRound);
-  uint32_t ybits[2][2];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const float2 x = unpack2(w[j]);
-    float2 y = magic;                                // code 0 when the sub-block has no scale
-    if (FAST || live) {                              // FAST: rc = 0 makes the reciprocal-based quotient 0, no branch needed
-      const float2 num = __fadd2_rn(x, em2);
-      float2 t = FAST ? div2_fast(num, es, rc) : make_float2(__fdiv_rn(num.x, es), __fdiv_rn(num.y, es));
-      t.x = fminf(fmaxf(t.x, 0.0f), 15.0f);          // clamp first: rounding is monotone and 0, 15 are integers
-      t.y = fminf(fmaxf(t.y, 0.0f), 15.0f);
-      y = __fadd2_rn(t, magic);                      // integer code now sits in the low mantissa bits
+  if (FAST) {
+    // The quotient (x + em) / es is monotone in x, so the sub-block's smallest and largest element bound every quotient;
+    // when both ends round into [0, 15] (the usual case: the 6-bit rounding of scale and offset moves them by a few
+    // percent of a step) the per-element clamp is left out. Same arithmetic as the loop, so the bound is exact.
+    const float t_lo = div1_fast(__fadd_rn(lo_raw, em), es, rc), t_hi = div1_fast(__fadd_rn(hi, em), es, rc);
+    const bool inside = t_lo >= -0.5f && t_hi < 15.5f;           // (a sub-block without a scale has rc = 0: both are 0)
+    if (__all_sync(0xFFFFFFFFu, inside)) {
+      q4k_elements<true, false>(w, es, em, rc, live, sink, cbytes);
+      return;
     }
-    const float2 c = __fadd2_rn(y, nmagic);
-    const float2 o = __ffma2_rn(es2, c, nem2);        // product exact: one rounding, as es*c - em
-    xhat[j & 3] = pack_bf16x2(o.x, o.y);
-    if ((j & 3) == 3 && out_ptr) out_ptr[j >> 2] = make_uint4(xhat[0], xhat[1], xhat[2], xhat[3]);   // stored as soon as complete
-    // the low byte of y's bit pattern is the code (the low byte of the rounding constant is zero)
-    ybits[j & 1][0] = __float_as_uint(y.x);
-    ybits[j & 1][1] = __float_as_uint(y.y);
-    if (j & 1) {
-      const uint32_t p01 = __byte_perm(ybits[0][0], ybits[0][1], 0x0040);
-      const uint32_t p23 = __byte_perm(ybits[1][0], ybits[1][1], 0x0040);
-      cbytes[j >> 1] = __byte_perm(p01, p23, 0x5410);             // codes 4k..4k+3, one per byte
+  }
+  q4k_elements<FAST, true>(w, es, em, rc, live, sink, cbytes);
+}
+
+// Everything after the load of one sub-block (16 words in w, slot c holding chunk c ^ perm of the sub-block; perm = 0
+// in the plain kernels): statistics, metadata, codes, dequantized values. `i` is the sub-block's index in the tensor.
+template <typename Sink>
+__device__ __forceinline__ void q4k_lane(const uint32_t (&w)[16], bool ok, int lane, const Sink sink, uint32_t perm,
+                                         uint4* __restrict__ codes, uint4* __restrict__ scales, int64_t i, uint32_t codes_smem = 0) {
+  __nv_bfloat162 mn = bits_bf2(w[0]), mx = bits_bf2(w[0]);
+#pragma unroll
+  for (int j = 1; j < 16; ++j) {
+    mn = __hmin2(mn, bits_bf2(w[j]));
+    mx = __hmax2(mx, bits_bf2(w[j]));
+  }
+  const float lo = fminf(bf16_lo(bf2_bits(mn)), bf16_hi(bf2_bits(mn)));
+  const float hi = fmaxf(bf16_lo(bf2_bits(mx)), bf16_hi(bf2_bits(mx)));
+  // the reciprocal-based division is exact away from the bottom of the FP32 range; a warp with a
+  // tiny but non-zero range or offset takes the IEEE divide instead
+  const float range = __fsub_rn(hi, fminf(lo, 0.0f)), offv = -fminf(lo, 0.0f);
+  const bool fast_ok = (range == 0.0f || (range >= 0x1p-60f && range <= 0x1p60f)) && (offv == 0.0f || (offv >= 0x1p-60f && offv <= 0x1p60f));
+  uint32_t cb[8], s6, m6;
+  __half d_h, dmin_h;
+  if (__all_sync(0xFFFFFFFFu, fast_ok)) q4k_subblock<true>(w, lo, hi, sink, cb, d_h, dmin_h, s6, m6);
+  else q4k_subblock<false>(w, lo, hi, sink, cb, d_h, dmin_h, s6, m6);
+  // cb[2c], cb[2c+1] hold the codes of slot c; put them back in chunk order (both lanes of a pair share perm)
+  if (perm & 1u) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      uint32_t t = cb[k]; cb[k] = cb[2 + k]; cb[2 + k] = t;
+      t = cb[4 + k]; cb[4 + k] = cb[6 + k]; cb[6 + k] = t;
+    }
+  }
+  if (perm & 2u) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { const uint32_t t = cb[k]; cb[k] = cb[4 + k]; cb[4 + k] = t; }
+  }
+  // code bytes: a 64-element chunk is the lane pair (2j, 2j+1); byte l = code[2j][l] | code[2j+1][l] << 4.
+  // cb[k] holds codes 4k..4k+3 one per byte. The even lane forms bytes 0-15, the odd lane bytes 16-31.
+  const bool odd = lane & 1;
+  uint32_t mine[4], theirs[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t send = odd ? cb[k] : cb[4 + k];            // what the partner needs from this lane
+    theirs[k] = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    mine[k] = odd ? cb[4 + k] : cb[k];
+  }
+  if (ok && codes) {
+    uint32_t o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o[k] = odd ? (theirs[k] | (mine[k] << 4)) : (mine[k] | (theirs[k] << 4));
+    // super-block = 8 lanes x 16 bytes = 128 bytes; chunk (lane/2 mod 4) owns 32 of them
+    if (codes_smem) st_shared_v4(codes_smem, o[0], o[1], o[2], o[3]);      // staged: leaves with the warp's bulk store
+    else codes[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  if (scales) {
+    const int b = lane & 7;                                       // sub-block within its super-block
+    uint32_t w0 = 0, w1 = 0, w2 = 0;                              // the 12 packed bytes as three words
+    if (b < 4) {
+      w0 = (s6 & 63u) << (8 * b);
+      w1 = (m6 & 63u) << (8 * b);
+    } else {
+      w0 = ((s6 >> 4) << 6) << (8 * (b - 4));
+      w1 = ((m6 >> 4) << 6) << (8 * (b - 4));
+      w2 = ((s6 & 15u) | ((m6 & 15u) << 4)) << (8 * (b - 4));
+    }
+#pragma unroll
+    for (int s = 1; s < 8; s <<= 1) {
+      w0 |= __shfl_xor_sync(0xFFFFFFFFu, w0, s);
+      w1 |= __shfl_xor_sync(0xFFFFFFFFu, w1, s);
+      w2 |= __shfl_xor_sync(0xFFFFFFFFu, w2, s);
+    }
+    if (ok && b == 0) {
+      const uint32_t hdr = static_cast<uint32_t>(__half_as_ushort(d_h)) | (static_cast<uint32_t>(__half_as_ushort(dmin_h)) << 16);
+      scales[i >> 3] = make_uint4(hdr, w0, w1, w2);
     }
   }
 }
@@ -298,63 +411,103 @@ __device__ __forceinline__ void qdq_q4k_body(const Loader& in, int64_t nsub, uin
       const uint4 v = ok ? in.chunk(4 * i + k) : make_uint4(0, 0, 0, 0);
       w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
     }
-    __nv_bfloat162 mn = bits_bf2(w[0]), mx = bits_bf2(w[0]);
-#pragma unroll
-    for (int j = 1; j < 16; ++j) {
-      mn = __hmin2(mn, bits_bf2(w[j]));
-      mx = __hmax2(mx, bits_bf2(w[j]));
+    q4k_lane(w, ok, lane, GlobalSink{(ok && out) ? out + 4 * i : nullptr}, 0u, codes, scales, i);
+  }
+}
+
+// ---- staged form --------------------------------------------------------------------------------------------------
+// The kernels above address global memory with a 64-byte stride between lanes (a lane owns a whole sub-block), which
+// costs the load/store data pipe several wavefronts per access: it is that pipe, at 76% of its peak, that holds the
+// plain kernel at 0.90 of the copy rate. Here the input travels global -> shared and the dequantized output shared ->
+// global as bulk asynchronous copies (a producer warp, a ring of mbarrier-guarded stages), and the lanes read and write
+// their 64-byte records in shared memory in a lane-dependent chunk order (slot c = chunk c ^ ((lane >> 1) & 3)) that
+// makes every 16-byte access bank-conflict free. Codes and metadata are already written with unit stride.
+constexpr int kQ4kTile = 256;                               // sub-blocks per tile: one per consumer thread, 16 KB of input
+constexpr int kQ4kStagesIn = 2, kQ4kStagesOut = 2;
+constexpr int kQ4kStagedThreads = kQ4kTile + 32;            // + the producer warp
+constexpr int kQ4kTileBytes = kQ4kTile * 64;
+constexpr int kQ4kCodeBytes = kQ4kTile * 16;                 // packed codes of one tile
+constexpr int kQ4kStagedSmem = (kQ4kStagesIn + kQ4kStagesOut) * kQ4kTileBytes + kQ4kStagesOut * kQ4kCodeBytes + 1024;
+
+__global__ void __launch_bounds__(kQ4kStagedThreads, 3) qdq_q4k_staged_kernel(const uint8_t* __restrict__ in, int64_t nsub,
+                                                                               uint8_t* __restrict__ out, uint4* __restrict__ codes,
+                                                                               uint4* __restrict__ scales, uint32_t* __restrict__ status) {
+  extern __shared__ uint8_t q4k_smem_raw[];
+  __shared__ uint64_t full[kQ4kStagesIn], empty[kQ4kStagesIn];
+  __shared__ int abort_flag;
+  const uint32_t base = (smem_u32(q4k_smem_raw) + 127u) & ~127u;
+  const uint32_t out_base = base + kQ4kStagesIn * kQ4kTileBytes;
+  const uint32_t code_base = out_base + kQ4kStagesOut * kQ4kTileBytes;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < kQ4kStagesIn; ++s) {
+      mbar_init(smem_u32(&full[s]), 1);
+      mbar_init(smem_u32(&empty[s]), kQ4kTile / 32);          // one arrival per consumer warp
     }
-    const float lo = fminf(bf16_lo(bf2_bits(mn)), bf16_hi(bf2_bits(mn)));
-    const float hi = fmaxf(bf16_lo(bf2_bits(mx)), bf16_hi(bf2_bits(mx)));
-    // the reciprocal-based division is exact away from the bottom of the FP32 range; a warp with a
-    // tiny but non-zero range or offset takes the IEEE divide instead
-    const float range = __fsub_rn(hi, fminf(lo, 0.0f)), offv = -fminf(lo, 0.0f);
-    const bool fast_ok = (range == 0.0f || (range >= 0x1p-60f && range <= 0x1p60f)) && (offv == 0.0f || (offv >= 0x1p-60f && offv <= 0x1p60f));
-    uint32_t cb[8], s6, m6;
-    __half d_h, dmin_h;
-    uint4* const out_ptr = (ok && out) ? out + 4 * i : nullptr;
-    if (__all_sync(0xFFFFFFFFu, fast_ok)) q4k_subblock<true>(w, lo, hi, out_ptr, cb, d_h, dmin_h, s6, m6);
-    else q4k_subblock<false>(w, lo, hi, out_ptr, cb, d_h, dmin_h, s6, m6);
-    // code bytes: a 64-element chunk is the lane pair (2j, 2j+1); byte l = code[2j][l] | code[2j+1][l] << 4.
-    // cb[k] holds codes 4k..4k+3 one per byte. The even lane forms bytes 0-15, the odd lane bytes 16-31.
-    const bool odd = lane & 1;
-    uint32_t mine[4], theirs[4];
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+  const int64_t ntiles = (nsub + kQ4kTile - 1) / kQ4kTile;
+  if (warp == kQ4kTile / 32) {
+    // ===== producer: one lane feeds the ring =====
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, &abort_flag, status)) break;
+        const int64_t first = t * kQ4kTile;
+        const uint32_t bytes = static_cast<uint32_t>(min(static_cast<int64_t>(kQ4kTile), nsub - first)) * 64u;
+        mbar_expect_tx(smem_u32(&full[stage]), bytes);
+        bulk_load(base + stage * kQ4kTileBytes, in + first * 64, bytes, smem_u32(&full[stage]));
+        if (++stage == kQ4kStagesIn) { stage = 0; phase ^= 1u; }
+      }
+    }
+    return;
+  }
+  // ===== consumers: thread tid owns sub-block tid of each tile =====
+  const uint32_t perm = (static_cast<uint32_t>(lane) >> 1) & 3u;
+  uint32_t stage = 0, phase = 0, local = 0;
+  for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++local) {
+    const int64_t i = t * kQ4kTile + tid;
+    const bool ok = i < nsub;
+    int got = 1;
+    if (lane == 0) got = mbar_wait(smem_u32(&full[stage]), phase, &abort_flag, status) ? 1 : 0;
+    got = __shfl_sync(0xFFFFFFFFu, got, 0);
+    if (!got) break;
+    uint32_t w[16];
+    const uint32_t rec = base + stage * kQ4kTileBytes + static_cast<uint32_t>(tid) * 64u;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const uint32_t send = odd ? cb[k] : cb[4 + k];            // what the partner needs from this lane
-      theirs[k] = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
-      mine[k] = odd ? cb[4 + k] : cb[k];
+      const uint4 v = ok ? ld_shared_v4(rec + ((static_cast<uint32_t>(k) ^ perm) << 4)) : make_uint4(0, 0, 0, 0);
+      w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
     }
-    if (ok && codes) {
-      uint32_t o[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) o[k] = odd ? (theirs[k] | (mine[k] << 4)) : (mine[k] | (theirs[k] << 4));
-      // super-block = 8 lanes x 16 bytes = 128 bytes; chunk (lane/2 mod 4) owns 32 of them
-      codes[i] = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-    if (scales) {
-      const int b = lane & 7;                                       // sub-block within its super-block
-      uint32_t w0 = 0, w1 = 0, w2 = 0;                              // the 12 packed bytes as three words
-      if (b < 4) {
-        w0 = (s6 & 63u) << (8 * b);
-        w1 = (m6 & 63u) << (8 * b);
-      } else {
-        w0 = ((s6 >> 4) << 6) << (8 * (b - 4));
-        w1 = ((m6 >> 4) << 6) << (8 * (b - 4));
-        w2 = ((s6 & 15u) | ((m6 & 15u) << 4)) << (8 * (b - 4));
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&empty[stage]));       // the record is in registers: the stage can be refilled
+    if (++stage == kQ4kStagesIn) { stage = 0; phase ^= 1u; }
+    // each warp stages and stores its own 32 records (2 KB of values, 512 bytes of codes): no block-wide synchronisation
+    // on the output side
+    const uint32_t obuf = out_base + (local & 1u) * kQ4kTileBytes + static_cast<uint32_t>(warp) * 2048u;
+    const uint32_t cbuf = code_base + (local & 1u) * kQ4kCodeBytes + static_cast<uint32_t>(warp) * 512u;
+    // the staging buffers about to be rewritten were the sources of the bulk stores this warp issued two tiles ago
+    if (lane == 0) bulk_wait_group_read<1>();
+    __syncwarp();
+    q4k_lane(w, ok, lane, SmemSink{obuf + static_cast<uint32_t>(lane) * 64u, perm, out != nullptr && ok}, perm, codes, scales, i,
+             cbuf + static_cast<uint32_t>(lane) * 16u);
+    fence_proxy_async_smem();                                  // generic-proxy writes -> visible to the bulk copies
+    __syncwarp();
+    if (lane == 0) {
+      const int64_t first = t * kQ4kTile + warp * 32;
+      const int64_t left = nsub - first;
+      if (left > 0) {
+        const uint32_t n = static_cast<uint32_t>(left < 32 ? left : 32);
+        if (out) bulk_store(out + first * 64, obuf, n * 64u);
+        if (codes) bulk_store(codes + first, cbuf, n * 16u);
       }
-#pragma unroll
-      for (int s = 1; s < 8; s <<= 1) {
-        w0 |= __shfl_xor_sync(0xFFFFFFFFu, w0, s);
-        w1 |= __shfl_xor_sync(0xFFFFFFFFu, w1, s);
-        w2 |= __shfl_xor_sync(0xFFFFFFFFu, w2, s);
-      }
-      if (ok && b == 0) {
-        const uint32_t hdr = static_cast<uint32_t>(__half_as_ushort(d_h)) | (static_cast<uint32_t>(__half_as_ushort(dmin_h)) << 16);
-        scales[i >> 3] = make_uint4(hdr, w0, w1, w2);
-      }
+      bulk_commit_group();
     }
   }
+  if (lane == 0) bulk_wait_group_all();                        // every store of this warp has left shared memory and landed
 }
 
 template <typename Loader>
@@ -648,6 +801,25 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
   return cudaGetLastError();
 }
 
+// The staged Q4_K kernel serves plain tensors large enough to fill its persistent grid several times over.
+template <typename Loader> static bool q4k_staged_applies(int64_t) { return false; }
+template <> bool q4k_staged_applies<PlainLoader>(int64_t nsub) { return nsub >= 4ll * kNumSMs * 2 * kQ4kTile; }
+
+static cudaError_t launch_q4k_staged(const QdqArgs& a, int64_t nsub, cudaStream_t st) {
+  static bool configured[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    if (cudaError_t e = cudaFuncSetAttribute(qdq_q4k_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQ4kStagedSmem)) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  const int64_t ntiles = (nsub + kQ4kTile - 1) / kQ4kTile;
+  const int grid = static_cast<int>(ntiles < 3ll * kNumSMs ? ntiles : 3ll * kNumSMs);
+  qdq_q4k_staged_kernel<<<grid, kQ4kStagedThreads, kQ4kStagedSmem, st>>>(static_cast<const uint8_t*>(a.in), nsub, static_cast<uint8_t*>(a.out),
+                                                                          static_cast<uint4*>(a.codes), static_cast<uint4*>(a.scales), nullptr);
+  return cudaGetLastError();
+}
+
 template <typename Loader>
 static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStream_t st) {
   const int64_t nelem = a.rows * a.cols;
@@ -667,6 +839,7 @@ static cudaError_t launch_qdq_with(const QdqArgs& a, const Loader& in, cudaStrea
         a.mxfp4_noclip ? 2 : 0, Nvfp4Speculation{a.spec.amax_accum, nullptr, nullptr});
   } else {
     const int64_t nsub = nelem / 32;
+    if (q4k_staged_applies<Loader>(nsub)) return launch_q4k_staged(a, nsub, st);
     qdq_q4k_kernel<Loader><<<capped_grid(nsub, 1, 32), kThreads, 0, st>>>(in, nsub, out, static_cast<uint4*>(a.codes),
                                                                           static_cast<uint4*>(a.scales));
   }

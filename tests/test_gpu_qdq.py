@@ -268,6 +268,23 @@ def test_q4k_worked_and_degenerate():
     _compare(api.FMT_Q4_K, f32_to_bits(tiny))
 
 
+def test_q4k_large_tensor_with_a_ragged_last_tile():
+    """Tensors of ten million elements and more take the Q4_K kernel that stages input and output through shared
+    memory with bulk asynchronous copies, 256 sub-blocks per tile. 1187 x 8448 has 313368 sub-blocks: a last tile of
+    24. All outputs, the codes-and-metadata-only form, and in place, bit for bit against the oracle."""
+    rows, cols = 1187, 8448
+    assert (rows * cols // 32) % 256 == 24
+    xb = torch_to_bits(synth.weight_with_outliers(rows, cols, seed=41))
+    g, o = _compare(api.FMT_Q4_K, xb)
+    x = bits_to_torch(xb, "cuda")
+    only = api.qf_qdq(api.FMT_Q4_K, x, want_out=False)
+    assert only["out"] is None and torch.equal(only["codes"], g["codes"]) and torch.equal(only["scales"], g["scales"])
+    inplace = api.qf_qdq(api.FMT_Q4_K, x, out=x)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(torch_to_bits(x), o["out"])
+    assert torch.equal(inplace["codes"], g["codes"])
+
+
 @pytest.mark.parametrize("fmt,name", FMTS)
 def test_two_runs_are_bitwise_identical(fmt, name):
     x = synth.weight_with_outliers(256, 4096, seed=9, device="cuda")
