@@ -801,9 +801,11 @@ cudaError_t launch_amax_to_float(const uint32_t* amax_bits, float* out, cudaStre
   return cudaGetLastError();
 }
 
-// The staged Q4_K kernel serves plain tensors large enough to fill its persistent grid several times over.
+// The staged Q4_K kernel serves plain tensors of 2^25 elements and more: at 2^24 (4096 x 4096: under five tiles per CTA) its
+// ramp-up and tail still cost more than the plain kernel's addressing (17.0 against 15.4 us); at 14336 x 4096 it wins
+// (51.5 against 54.6 us, sustained).
 template <typename Loader> static bool q4k_staged_applies(int64_t) { return false; }
-template <> bool q4k_staged_applies<PlainLoader>(int64_t nsub) { return nsub >= 4ll * kNumSMs * 2 * kQ4kTile; }
+template <> bool q4k_staged_applies<PlainLoader>(int64_t nsub) { return nsub >= (1ll << 20); }
 
 static cudaError_t launch_q4k_staged(const QdqArgs& a, int64_t nsub, cudaStream_t st) {
   static bool configured[64] = {false};

@@ -269,11 +269,11 @@ def test_q4k_worked_and_degenerate():
 
 
 def test_q4k_large_tensor_with_a_ragged_last_tile():
-    """Tensors of ten million elements and more take the Q4_K kernel that stages input and output through shared
-    memory with bulk asynchronous copies, 256 sub-blocks per tile. 1187 x 8448 has 313368 sub-blocks: a last tile of
-    24. All outputs, the codes-and-metadata-only form, and in place, bit for bit against the oracle."""
-    rows, cols = 1187, 8448
-    assert (rows * cols // 32) % 256 == 24
+    """Tensors of 2^25 elements and more take the Q4_K kernel that stages input and output through shared memory with
+    bulk asynchronous copies, 256 sub-blocks per tile. 4099 x 8448 has 1082136 sub-blocks: a last tile of 24. All
+    outputs, the codes-and-metadata-only form, and in place, bit for bit against the oracle."""
+    rows, cols = 4099, 8448
+    assert (rows * cols // 32) % 256 == 24 and rows * cols >= 2 ** 25
     xb = torch_to_bits(synth.weight_with_outliers(rows, cols, seed=41))
     g, o = _compare(api.FMT_Q4_K, xb)
     x = bits_to_torch(xb, "cuda")
